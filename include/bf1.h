@@ -1,0 +1,146 @@
+/*
+ * bf1.h -- C ABI of the BF1 causal dyadic block-sparse attention forward (prefill) library
+ *          for NVIDIA B200 (sm_100a).
+ *
+ * The operator (paper Section 3.1): a sequence of n tokens is cut into B = ceil(n / b)
+ * blocks of width b.  Query block j attends, with exact softmax, to the keys of the blocks
+ *
+ *        P(j) = {j, j-1, j-2, 0} u {j - 2^r : r >= 2}        (Eq. 1)
+ *
+ * with invalid and duplicate indices removed; inside the self block the token-level causal
+ * triangle applies, every other selected block is strictly earlier and is read in full.
+ * No score bias is used.  Proposition 1 bounds |P(j)| by 4 + floor(log2 j), which makes the
+ * selected token pairs O(n log n).
+ *
+ * Conventions for every entry point
+ *   - C linkage, plain pointers and sizes, int status return (bf1_status); no exceptions.
+ *   - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are
+ *     ordinary host memory.  The library allocates no device memory.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream) and return without synchronising.  Host-checkable argument errors are
+ *     reported before anything is launched.  Errors that only the device can see are
+ *     OR-ed into the route's `status` word (see BF1_DEV_* below), never a trap.
+ *   - Tensors are packed over the batch ("varlen"): Q and O are [T, Hq, d], K and V are
+ *     [T, Hkv, d], bf16, row-major, T = total tokens; sequence s owns token rows
+ *     cu_seqlens[s] .. cu_seqlens[s+1]-1.  With equal lengths this is [B, n, H, d].
+ *     LSE is fp32 [Hq, T].  Every sequence is cut into blocks from its own first token and
+ *     never attends across a sequence boundary.
+ *   - GQA: Hq = G * Hkv; query head h reads KV head floor(h / G) (the paper gives only the
+ *     head counts, Section 4.1; this is the usual grouped convention).
+ *   - Base pointers of Q, K, V, O must be 16-byte aligned.
+ *   - Supported geometry: b = 64, d in {64, 128}, G = 2 (Section 4.1's 16 query / 8 KV
+ *     heads, Section 3.1's b = 64).  Anything else returns BF1_ERR_UNSUPPORTED.
+ */
+#ifndef BF1_H_
+#define BF1_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BF1_OK = 0,
+    BF1_ERR_INVALID_ARG = -1,   /* null pointer, negative size, misaligned pointer, ...   */
+    BF1_ERR_UNSUPPORTED = -2,   /* geometry outside the supported set                     */
+    BF1_ERR_CAPACITY = -3,      /* route buffers too small for this batch                 */
+    BF1_ERR_CUDA = -4,          /* a CUDA runtime / driver call failed                    */
+    BF1_ERR_NO_DEVICE = -5      /* no usable sm_100 device                                */
+} bf1_status;
+
+/* Bits OR-ed into *route.status by device code. */
+enum {
+    BF1_DEV_BAD_SEQLENS = 1,    /* cu_seqlens not non-decreasing from 0 to total_tokens,
+                                   or a sequence longer than max_seqlen                   */
+    BF1_DEV_CAPACITY = 2,       /* more query blocks, or a longer list, than the buffers  */
+    BF1_DEV_WAIT_TIMEOUT = 4,   /* a bounded on-chip wait gave up (should never happen)   */
+    BF1_DEV_BAD_ROUTE = 8       /* attention kernel met a list entry outside [0, j]       */
+};
+
+/* Route parameters.  The paper's reported configuration (Section 3.1) is
+ * {64, 2, 1, 1}: two local predecessor blocks, the global first block, dyadic
+ * predecessors.  `dyadic` adds j - 2^k for every k >= 0 with j - 2^k >= 0; with
+ * local_blocks = 2 this is Eq. 1's "r >= 2" set, because 2^0 and 2^1 are the local blocks. */
+typedef struct {
+    int32_t block;         /* b; must be 64                                              */
+    int32_t local_blocks;  /* W >= 0                                                     */
+    int32_t global_first;  /* 0 or 1                                                     */
+    int32_t dyadic;        /* 0 or 1                                                     */
+} bf1_route_cfg;
+
+/* A planned route: for every query block of every sequence, the ascending list of KV
+ * block indices it reads (sequence-local; the last entry is the query block itself), the
+ * list length, and the number of selected token pairs (Proposition 1's accounting: a
+ * non-self block gives rows*b pairs, the self block rows*(rows+1)/2, rows = tokens in the
+ * query block).  Query blocks are numbered sequence by sequence ("slots").
+ * The two capacities are host values; every pointer is device memory owned by the caller. */
+typedef struct {
+    int32_t  capacity_qblocks; /* slots available in the arrays below                     */
+    int32_t  max_degree;       /* row pitch of kv_idx                                     */
+    int32_t *qb_seq;           /* [capacity] sequence of the slot                         */
+    int32_t *qb_block;         /* [capacity] block index j inside that sequence           */
+    int32_t *kv_count;         /* [capacity] |P(j)|                                       */
+    int32_t *kv_idx;           /* [capacity, max_degree] ascending; unused entries = -1   */
+    int32_t *pair_count;       /* [capacity] selected token pairs of the slot             */
+    int32_t *order;            /* [capacity] slots sorted by descending kv_count: the
+                                  order in which the attention kernel hands out work      */
+    int64_t *total_pairs;      /* [1] sum of pair_count                                   */
+    int32_t *num_qblocks;      /* [1] slots actually used                                 */
+    int32_t *status;           /* [1] BF1_DEV_* bits; 0 = fine.  Written (not OR-ed) by
+                                  bf1_plan_route, OR-ed by the attention entry points     */
+} bf1_route;
+
+/* Host-only helper: how large the route arrays must be for a batch of `batch` sequences,
+ * `total_tokens` tokens in all, none longer than `max_seqlen`.  capacity_qblocks is an
+ * upper bound on sum_s ceil(n_s / b); max_degree is the largest |P(j)| any block of a
+ * sequence of max_seqlen tokens has (Proposition 1).  Touches no device. */
+int bf1_route_capacity(int32_t batch, int64_t total_tokens, int32_t max_seqlen,
+                       const bf1_route_cfg *cfg /* host */,
+                       int32_t *capacity_qblocks /* host out */, int32_t *max_degree /* host out */);
+
+/* Eq. 1 on the device: fills every array of `out` from cu_seqlens.  One small kernel; meant
+ * to run once per (sequence lengths, cfg) and be reused by every layer.
+ *   cu_seqlens_dev  [batch+1] int32 device, cu_seqlens[0] = 0, cu_seqlens[batch] = total_tokens
+ *   out             host struct holding device pointers (see bf1_route)
+ * Device-side validation failures set *out->status and leave num_qblocks = 0. */
+int bf1_plan_route(const int32_t *cu_seqlens_dev, int32_t batch, int64_t total_tokens,
+                   int32_t max_seqlen, const bf1_route_cfg *cfg /* host */,
+                   const bf1_route *out /* host struct, device arrays */, void *stream);
+
+/* BF1 forward (Section 3.1): for every query block, online-softmax attention over exactly
+ * the KV blocks its list names, causal triangle on the self block.
+ *   q, k, v   device bf16, [T, hq, d], [T, hkv, d], [T, hkv, d]
+ *   softmax_scale  scores are scale * <q, k>; <= 0 selects 1 / sqrt(d)
+ *   route     a route planned for the same cu_seqlens (any ascending lists whose last
+ *             entry is the query block itself are accepted, so other block-sparse causal
+ *             routes can be run through the same kernel)
+ *   o         device bf16 [T, hq, d], written for every token row
+ *   lse       device fp32 [hq, T]: natural log of the sum of exp(scaled scores) over the
+ *             selected keys
+ * Rows of o/lse outside every sequence are not touched. */
+int bf1_attn_fwd(const void *q, const void *k, const void *v, const int32_t *cu_seqlens_dev,
+                 int32_t batch, int64_t total_tokens, int32_t max_seqlen, int32_t hq,
+                 int32_t hkv, int32_t d, float softmax_scale, const bf1_route *route /* host */,
+                 void *o, float *lse, void *stream);
+
+/* Dense causal attention through the same kernel (every predecessor block selected):
+ * the paper's dense comparator (Section 4.3) and its dense-path equivalence gate
+ * (Section 4.2).  Arguments as bf1_attn_fwd without the route; `status_dev` is an optional
+ * [1] int32 device word for BF1_DEV_* bits (may be NULL). */
+int bf1_dense_causal_fwd(const void *q, const void *k, const void *v,
+                         const int32_t *cu_seqlens_dev, int32_t batch, int64_t total_tokens,
+                         int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d,
+                         float softmax_scale, void *o, float *lse, int32_t *status_dev,
+                         void *stream);
+
+/* Message for the last non-OK status returned on the calling thread ("" if none). */
+const char *bf1_last_error(void);
+
+/* Library version, for the binding's sanity check. */
+int bf1_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BF1_H_ */

@@ -1,0 +1,201 @@
+"""Thin Python binding of the BF1 C-ABI library (argument marshalling only).
+
+Every step of the operator runs in the library's CUDA kernels.  PyTorch is used for device
+memory, streams and nothing else.  There is no CPU or PyTorch fallback: if the shared
+library cannot be built or loaded, importing callers get an exception.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+BF1_OK = 0
+DEV_BAD_SEQLENS, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_ROUTE = 1, 2, 4, 8
+
+EXPORTS = ("bf1_route_capacity", "bf1_plan_route", "bf1_attn_fwd", "bf1_dense_causal_fwd",
+           "bf1_last_error", "bf1_version")
+
+
+class RouteCfg(ctypes.Structure):
+    """Mirror of bf1_route_cfg.  Defaults: the paper's reported configuration (Section 3.1)."""
+    _fields_ = [("block", ctypes.c_int32), ("local_blocks", ctypes.c_int32),
+                ("global_first", ctypes.c_int32), ("dyadic", ctypes.c_int32)]
+
+    def __init__(self, block: int = 64, local_blocks: int = 2, global_first: int = 1, dyadic: int = 1):
+        super().__init__(block, local_blocks, global_first, dyadic)
+
+
+class _RouteC(ctypes.Structure):
+    """Mirror of bf1_route."""
+    _fields_ = [("capacity_qblocks", ctypes.c_int32), ("max_degree", ctypes.c_int32),
+                ("qb_seq", ctypes.c_void_p), ("qb_block", ctypes.c_void_p),
+                ("kv_count", ctypes.c_void_p), ("kv_idx", ctypes.c_void_p),
+                ("pair_count", ctypes.c_void_p), ("order", ctypes.c_void_p),
+                ("total_pairs", ctypes.c_void_p), ("num_qblocks", ctypes.c_void_p),
+                ("status", ctypes.c_void_p)]
+
+
+class Bf1Error(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("bf1 error %d: %s" % (code, msg))
+        self.code = code
+
+
+_lib = None
+
+
+def load():
+    """Load (building first if needed) libbf1.so and declare its signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    L = ctypes.CDLL(path)
+    i32, i64, vp, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float
+    L.bf1_route_capacity.restype = ctypes.c_int
+    L.bf1_route_capacity.argtypes = [i32, i64, i32, ctypes.POINTER(RouteCfg), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.bf1_plan_route.restype = ctypes.c_int
+    L.bf1_plan_route.argtypes = [vp, i32, i64, i32, ctypes.POINTER(RouteCfg), ctypes.POINTER(_RouteC), vp]
+    L.bf1_attn_fwd.restype = ctypes.c_int
+    L.bf1_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(_RouteC), vp, vp, vp]
+    L.bf1_dense_causal_fwd.restype = ctypes.c_int
+    L.bf1_dense_causal_fwd.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, vp, vp, vp, vp]
+    L.bf1_last_error.restype = ctypes.c_char_p
+    L.bf1_last_error.argtypes = []
+    L.bf1_version.restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def _check(rc: int):
+    if rc != BF1_OK:
+        raise Bf1Error(rc, load().bf1_last_error().decode())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def route_capacity(batch: int, total_tokens: int, max_seqlen: int, cfg: Optional[RouteCfg] = None):
+    """(capacity_qblocks, max_degree) for a batch; host only."""
+    cfg = cfg or RouteCfg()
+    cap, deg = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(load().bf1_route_capacity(batch, total_tokens, max_seqlen, ctypes.byref(cfg),
+                                     ctypes.byref(cap), ctypes.byref(deg)))
+    return cap.value, deg.value
+
+
+@dataclass
+class Route:
+    """Device arrays of a planned route plus the C struct that points at them."""
+    cfg: RouteCfg
+    capacity_qblocks: int
+    max_degree: int
+    qb_seq: torch.Tensor
+    qb_block: torch.Tensor
+    kv_count: torch.Tensor
+    kv_idx: torch.Tensor
+    pair_count: torch.Tensor
+    order: torch.Tensor
+    total_pairs: torch.Tensor
+    num_qblocks: torch.Tensor
+    status: torch.Tensor
+    c: _RouteC = None
+
+    @staticmethod
+    def empty(capacity_qblocks: int, max_degree: int, device, cfg: Optional[RouteCfg] = None) -> "Route":
+        i32 = dict(dtype=torch.int32, device=device)
+        r = Route(cfg=cfg or RouteCfg(), capacity_qblocks=capacity_qblocks, max_degree=max_degree,
+                  qb_seq=torch.empty(capacity_qblocks, **i32), qb_block=torch.empty(capacity_qblocks, **i32),
+                  kv_count=torch.empty(capacity_qblocks, **i32),
+                  kv_idx=torch.empty((capacity_qblocks, max_degree), **i32),
+                  pair_count=torch.empty(capacity_qblocks, **i32), order=torch.empty(capacity_qblocks, **i32),
+                  total_pairs=torch.zeros(1, dtype=torch.int64, device=device),
+                  num_qblocks=torch.zeros(1, **i32), status=torch.zeros(1, **i32))
+        r.c = _RouteC(capacity_qblocks, max_degree, r.qb_seq.data_ptr(), r.qb_block.data_ptr(),
+                      r.kv_count.data_ptr(), r.kv_idx.data_ptr(), r.pair_count.data_ptr(), r.order.data_ptr(),
+                      r.total_pairs.data_ptr(), r.num_qblocks.data_ptr(), r.status.data_ptr())
+        return r
+
+    def check_status(self):
+        """Synchronising read of the device status word; raises if any BF1_DEV_* bit is set."""
+        st = int(self.status.item())
+        if st:
+            raise Bf1Error(-100, "device status 0x%x" % st)
+
+
+def plan_route(cu_seqlens: torch.Tensor, max_seqlen: int, cfg: Optional[RouteCfg] = None,
+               route: Optional[Route] = None, stream=None) -> Route:
+    """bf1_plan_route: Eq. 1 lists for every query block of the packed batch."""
+    cfg = cfg or RouteCfg()
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    batch = cu_seqlens.numel() - 1
+    total = getattr(cu_seqlens, "_bf1_total", None)
+    if total is None:
+        total = int(cu_seqlens[-1].item())
+    if route is None:
+        cap, deg = route_capacity(batch, total, max_seqlen, cfg)
+        route = Route.empty(cap, deg, cu_seqlens.device, cfg)
+    _check(load().bf1_plan_route(cu_seqlens.data_ptr(), batch, total, max_seqlen, ctypes.byref(cfg),
+                                 ctypes.byref(route.c), _stream_ptr(stream)))
+    route.cfg = cfg
+    return route
+
+
+def _check_qkv(q, k, v):
+    for t in (q, k, v):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 3
+    T, hq, d = q.shape
+    assert k.shape == v.shape and k.shape[0] == T and k.shape[2] == d
+    return T, hq, k.shape[1], d
+
+
+def attn_fwd(q, k, v, cu_seqlens, max_seqlen: int, route: Route, scale: Optional[float] = None,
+             out=None, lse=None, stream=None):
+    """bf1_attn_fwd.  q [T, hq, d], k/v [T, hkv, d] bf16 CUDA -> (o [T, hq, d] bf16, lse [hq, T] fp32)."""
+    T, hq, hkv, d = _check_qkv(q, k, v)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((hq, T), dtype=torch.float32, device=q.device)
+    _check(load().bf1_attn_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), cu_seqlens.data_ptr(),
+                               cu_seqlens.numel() - 1, T, max_seqlen, hq, hkv, d,
+                               float(scale) if scale else 0.0, ctypes.byref(route.c), out.data_ptr(),
+                               lse.data_ptr(), _stream_ptr(stream)))
+    return out, lse
+
+
+def dense_causal_fwd(q, k, v, cu_seqlens, max_seqlen: int, scale: Optional[float] = None, out=None,
+                     lse=None, status=None, stream=None):
+    """bf1_dense_causal_fwd: plain causal attention through the same kernel."""
+    T, hq, hkv, d = _check_qkv(q, k, v)
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((hq, T), dtype=torch.float32, device=q.device)
+    _check(load().bf1_dense_causal_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), cu_seqlens.data_ptr(),
+                                       cu_seqlens.numel() - 1, T, max_seqlen, hq, hkv, d,
+                                       float(scale) if scale else 0.0, out.data_ptr(), lse.data_ptr(),
+                                       status.data_ptr() if status is not None else None,
+                                       _stream_ptr(stream)))
+    return out, lse
+
+
+def cu_seqlens_tensor(seqlens: Sequence[int], device) -> torch.Tensor:
+    cu = [0]
+    for n in seqlens:
+        cu.append(cu[-1] + int(n))
+    t = torch.tensor(cu, dtype=torch.int32, device=device)
+    t._bf1_total = cu[-1]   # host copy of the total, saves a device sync in plan_route
+    return t
+
+
+def default_scale(d: int) -> float:
+    return 1.0 / math.sqrt(d)
