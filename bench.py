@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the BF1 forward hot path on B200.
+
+One step = one route plan (bf1_plan_route) followed by eight back-to-back bf1_attn_fwd
+calls on eight independent sets of Q/K/V at n = 32768, 16 query / 8 KV heads, d = 128:
+the eight retrofitted layers of the paper's model sharing one plan (Section 3.4, 4.3).
+The eight input sets together are ~2.1 GB, far larger than L2, so no flush is needed.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is selected-pair TFLOP/s = 4 * d * pairs * Hq * layers
+/ step time, summed over ranks (each rank runs its own independent copy: weak scaling, no
+collective on the data path).  `--impl reference` times the CPU oracle on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import bf1_inputs as I  # noqa: E402
+
+WORKLOAD = "qwen_32k"
+LAYERS = 8
+METRIC = "bf1_fwd_prefill_selected_pair_tflops"
+UNIT = "TFLOP/s"
+
+
+# ---- closed-form work accounting (Proposition 1; no oracle needed) -------------------------
+def degree(j: int) -> int:
+    if j <= 3:
+        return j + 1
+    return int(math.floor(math.log2(j))) + 3 - (1 if j & (j - 1) == 0 else 0)
+
+
+def row_pairs(i: int, b: int = 64) -> int:
+    return b * (degree(i // b) - 1) + (i % b) + 1
+
+
+def selected_pairs(n: int, b: int = 64) -> int:
+    total = 0
+    nb = (n + b - 1) // b
+    for j in range(nb):
+        rows = min(b, n - j * b)
+        total += rows * b * (degree(j) - 1) + rows * (rows + 1) // 2
+    return total
+
+
+def flops(pairs: int, d: int, hq: int) -> float:
+    return 4.0 * d * pairs * hq
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p.get("bf16_tflops_sustained"),
+                "hbm_gbs": p["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# ---- clock sampling through NVML (read-only) ------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.stop_flag, self.thread, self.max_mhz = [], set(), False, None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        while not self.stop_flag:
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                r = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if r & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def start(self):
+        if self.nv:
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
+
+    def stop(self):
+        self.stop_flag = True
+        if self.thread:
+            self.thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---- reference arm / cpu baseline: the oracle on the host cores ------------------------------
+def oracle_rate(w, q, k, v, target_s: float):
+    """Time the CPU oracle on a strided row sample sized for ~target_s seconds.
+    Returns (TFLOP/s, seconds, description, threads)."""
+    from oracle import bf1_oracle as O
+    n = w.seqlens[0]
+    cfg = O.cfg(w.block, w.local_blocks, w.global_first, w.dyadic)
+    probe = list(range(0, n, 32))
+    t0 = time.perf_counter()
+    O.attn_route(cfg, q, k, v, w.cu_seqlens(), rows=probe)
+    t_probe = time.perf_counter() - t0
+    full_est = t_probe * sum(row_pairs(i) for i in range(0, n, 16)) * 16 / max(sum(row_pairs(i) for i in probe), 1)
+    stride = max(1, int(math.ceil(full_est / target_s)))
+    rows = list(range(0, n, stride))
+    t0 = time.perf_counter()
+    O.attn_route(cfg, q, k, v, w.cu_seqlens(), rows=rows)
+    dt = time.perf_counter() - t0
+    fl = flops(sum(row_pairs(i) for i in rows), w.d, w.hq)
+    return fl / dt / 1e12, dt, "every %d-th token row of one %s layer (%d rows x %d heads)" % (
+        stride, w.name, len(rows), w.hq), O.threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = I.WORKLOADS[WORKLOAD]
+    q, k, v = I.draw_qkv(w)
+    vals, secs, desc, thr = [], [], "", 1
+    for s in range(args.warmup + args.steps):
+        val, dt, desc, thr = oracle_rate(w, q, k, v, target_s=min(2.0, 150.0 / (args.warmup + args.steps)))
+        if s >= args.warmup:
+            vals.append(val)
+            secs.append(dt)
+    value = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "%s x %d layers, 16q/8kv d128 b64, BF1 route" % (WORKLOAD, LAYERS),
+                       "sample_per_step": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---- our arm -----------------------------------------------------------------------------------
+def time_region(fn, reps, stream):
+    """Median CUDA-event time (ms) of fn() over reps runs."""
+    out = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        e1.synchronize()
+        out.append(e0.elapsed_time(e1))
+    return statistics.median(out)
+
+
+def sweep(bf1, dev):
+    """BF1 vs the library's dense-causal mode, per layer, with the paper's protocol (Section
+    4.3): 5 warm-ups, 30 repetitions, two opposite pattern orders, median of the order medians."""
+    out = []
+    for name in ("qwen_2k", "qwen_4k", "qwen_8k", "qwen_16k", "qwen_32k"):
+        w = I.WORKLOADS[name]
+        q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+        cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+        route = bf1.plan_route(cu, w.max_seqlen)
+        o = torch.empty_like(q)
+        lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
+        stream = torch.cuda.current_stream()
+        f_s = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
+        f_d = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse)
+        meds = {"bf1": [], "dense": []}
+        for order in (("dense", "bf1"), ("bf1", "dense")):
+            for which in order:
+                f = f_s if which == "bf1" else f_d
+                for _ in range(5):
+                    f()
+                meds[which].append(time_region(f, 30, stream))
+        ms_s, ms_d = statistics.median(meds["bf1"]), statistics.median(meds["dense"])
+        n = w.seqlens[0]
+        pairs = selected_pairs(n)
+        out.append({"n": n, "bf1_ms": round(ms_s, 5), "dense_ms": round(ms_d, 5), "speedup": round(ms_d / ms_s, 3),
+                    "bf1_tflops": round(flops(pairs, w.d, w.hq) / ms_s / 1e9, 1),
+                    "dense_tflops": round(flops(n * (n + 1) // 2, w.d, w.hq) / ms_d / 1e9, 1),
+                    "pair_reduction": round(n * (n + 1) / 2 / pairs, 3), "inputs": "L2-warm (same buffers re-run)"})
+        del q, k, v, o, lse
+    return out
+
+
+def run_ours(args):
+    import paper_2608_20427_b200 as bf1
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    bf1.load()
+
+    w = I.WORKLOADS[WORKLOAD]
+    n, T = w.seqlens[0], w.total_tokens
+    pairs = selected_pairs(n)
+    layer_flops = flops(pairs, w.d, w.hq)
+    step_flops = layer_flops * LAYERS
+
+    # eight independent layers' inputs: host (pinned) and device copies
+    host = []
+    for layer in range(LAYERS):
+        host.append(tuple(t.pin_memory() for t in I.draw_qkv(w, layer=layer + rank * LAYERS)))
+    devb = [tuple(t.to(dev) for t in h) for h in host]
+    outs = [torch.empty((T, w.hq, w.d), dtype=torch.bfloat16, device=dev) for _ in range(LAYERS)]
+    lses = [torch.empty((w.hq, T), dtype=torch.float32, device=dev) for _ in range(LAYERS)]
+    cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+    cap, deg = bf1.route_capacity(1, T, n)
+    route = bf1.Route.empty(cap, deg, dev)
+    stream = torch.cuda.current_stream()
+
+    attn_ms = []   # per step: time of the eight attention launches alone
+
+    def step(record=False):
+        bf1.plan_route(cu, n, route=route)
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        for layer in range(LAYERS):
+            q, k, v = devb[layer]
+            bf1.attn_fwd(q, k, v, cu, n, route, out=outs[layer], lse=lses[layer])
+        if record:
+            e1.record(stream)
+            attn_ms.append((e0, e1))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step(record=True)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    route.check_status()
+    assert int(route.total_pairs.item()) == pairs
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_ms) / LAYERS
+
+    # ---- end to end: pinned host buffers -> device -> kernels -> host, every step
+    o_host = [torch.empty((T, w.hq, w.d), dtype=torch.bfloat16).pin_memory() for _ in range(LAYERS)]
+    l_host = [torch.empty((w.hq, T), dtype=torch.float32).pin_memory() for _ in range(LAYERS)]
+    h2d = sum(t.numel() * t.element_size() for h in host for t in h)
+    d2h = sum(t.numel() * t.element_size() for t in o_host + l_host)
+
+    def e2e_step():
+        bf1.plan_route(cu, n, route=route)
+        for layer in range(LAYERS):
+            for src, dst in zip(host[layer], devb[layer]):
+                dst.copy_(src, non_blocking=True)
+            q, k, v = devb[layer]
+            bf1.attn_fwd(q, k, v, cu, n, route, out=outs[layer], lse=lses[layer])
+            o_host[layer].copy_(outs[layer], non_blocking=True)
+            l_host[layer].copy_(lses[layer], non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * step_flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    achieved = layer_flops / (kern_ms * 1e-3) / 1e12
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "attn_fwd_qwen_32k_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get("dram_bytes_per_launch")
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "%s x %d layers per step (one plan + %d bf1_attn_fwd), B=1 n=32768 16q/8kv d128 b64, "
+                               "BF1 route (W=2, block 0, dyadic)" % (WORKLOAD, LAYERS, LAYERS),
+                   "ms_per_layer": ms_per_step / LAYERS, "selected_pairs_per_layer": pairs,
+                   "l2": "inputs larger than L2 (8 layers x 268 MB rotate)", "timing": "CUDA events, max over ranks"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
+        "gpu_launches": args.steps * (LAYERS + 1),
+        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel<128>", "achieved": achieved,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                     "peak_source": "%s burst bf16 (MEASURED_PEAKS.json)" % peaks["source"],
+                     "frac_of_sustained": (achieved / peaks["bf16_tflops_sustained"]) if peaks["bf16_tflops_sustained"] else None,
+                     "traffic": traffic, "algorithmic_flops_per_launch": layer_flops,
+                     "kernel_ms_per_launch": kern_ms},
+    }
+    if not args.no_sweep and world == 1:
+        line["sweep"] = sweep(bf1, dev)
+    if not args.no_cpu and world == 1:
+        q, k, v = I.draw_qkv(w)
+        val, dt, desc, thr = oracle_rate(w, q, k, v, target_s=15.0)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc,
+                                "seconds": dt}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
