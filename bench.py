@@ -205,6 +205,32 @@ def sweep(bf1, dev):
     return out
 
 
+def run_single(args):
+    """A few plain launches of one mode on one named workload (what the ncu captures run)."""
+    import paper_2608_20427_b200 as bf1
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = I.WORKLOADS[args.single]
+    q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+    cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+    route = bf1.plan_route(cu, w.max_seqlen)
+    o = torch.empty_like(q)
+    lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    if args.mode == "dense":
+        f = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse)
+        pairs = sum(n * (n + 1) // 2 for n in w.seqlens)
+    else:
+        f = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
+        pairs = sum(selected_pairs(n) for n in w.seqlens)
+    for _ in range(args.warmup):
+        f()
+    ms = time_region(f, args.steps, stream)
+    route.check_status()
+    print(json.dumps({"single": args.single, "mode": args.mode, "ms": ms, "steps": args.steps,
+                      "tflops": flops(pairs, w.d, w.hq) / ms / 1e9}))
+
+
 def run_ours(args):
     import paper_2608_20427_b200 as bf1
     rank = int(os.environ.get("RANK", "0"))
@@ -363,8 +389,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--single", default=None, choices=sorted(I.WORKLOADS),
+                    help="only time `--steps` launches of one workload (used for profiling)")
+    ap.add_argument("--mode", default="bf1", choices=["bf1", "dense"])
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.single:
+        run_single(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

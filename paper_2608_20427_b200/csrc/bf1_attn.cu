@@ -4,24 +4,34 @@
 // heads that share the KV head are stacked into one M = 128 tile (rows 0..63: first head,
 // rows 64..127: second head), because they read the same K/V blocks through the same route
 // list (the route is per block and the same for all heads, Section 3.1).  For every entry p
-// of the unit's list the kernel
-//   TMA-loads K[p], V[p] (64 x d each, 128-byte swizzle) into shared memory,
-//   S = Q K[p]^T        tcgen05.mma, operands in shared memory, fp32 accumulator in TMEM,
-//   online softmax      one thread per row: tcgen05.ld S, mask (self block only), running
-//                       max / sum in the exp2 domain, P -> bf16 -> tcgen05.st over S,
-//   O += P V[p]         tcgen05.mma with P read from TMEM and V from shared memory,
-// and finally writes O / l as bf16 and LSE = max + ln(sum) as fp32.
+// of the unit's list ("tile"):
+//   S = Q K[p]^T        tcgen05.mma, Q and K[p] in shared memory (TMA, 128-byte swizzle),
+//                       fp32 accumulator in tensor memory (two S buffers, ping-pong),
+//   online softmax      one thread per row: tcgen05.ld S, causal mask on the self block only,
+//                       running max / sum in the exp2 domain, P -> bf16 -> tcgen05.st over S,
+//   O += P V[p]         tcgen05.mma with P read from tensor memory and V from shared memory,
+// then O / l is written as bf16 and LSE = max + ln(sum) as fp32.
 // With `dense = 1` the list is replaced by 0..j: plain causal attention through the same code.
+//
+// The kernel is persistent (two CTAs per SM, each walking a strided share of the units in
+// longest-list-first order) and warp specialised:
+//   warp 0     TMA producer: Q once per unit, then K and V tiles through a ring of 16 KB slots
+//              in the order the MMAs consume them (K0, K1, V0, K2, V1, ...),
+//   warp 1     MMA issuer: S(g+1) is issued before PV(g), so the tensor pipe works on the next
+//              tile's scores and the previous tile's PV while the softmax warps are busy,
+//   warps 2-5  softmax + epilogue, one thread per tile row.
+// All hand-offs are mbarriers; every wait is bounded (see mbar_wait).
 #include <cuda.h>
 
 #include "bf1_common.cuh"
 
 namespace bf1 {
 
-constexpr int kBlock = 64;      // b: tokens per block
-constexpr int kRows = 128;      // MMA M: 2 query heads x 64 tokens
-constexpr int kThreads = 128;   // one thread per tile row
-constexpr int kStages = 2;      // K/V shared-memory ring
+constexpr int kBlock = 64;            // b: tokens per block
+constexpr int kRows = 128;            // MMA M: 2 query heads x 64 tokens
+constexpr int kThreads = 192;         // 6 warps
+constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row
+                                            // maximum grows by more than 2^8
 
 struct AttnArgs {
     const int32_t* cu_seqlens;
@@ -35,256 +45,348 @@ struct AttnArgs {
     const int32_t* qb_block;
     const int32_t* kv_count;
     const int32_t* kv_idx;
+    const int32_t* order;  // may be null
     const int32_t* num_qblocks;
     int32_t max_degree;
+    int32_t capacity;
     int32_t* status;       // may be null in dense mode
     __nv_bfloat16* o;
     float* lse;
 };
 
 template <int D>
-struct Smem {
+struct Cfg {
     static constexpr int kChunks = D / 64;                 // 128-byte column chunks per row
     static constexpr int kQBytes = kRows * D * 2;          // 32 KB at d = 128
-    static constexpr int kKVBytes = kBlock * D * 2;        // 16 KB at d = 128
+    static constexpr int kTileBytes = kBlock * D * 2;      // one K or V block: 16 KB at d = 128
+    static constexpr int kRing = (D == 128) ? 5 : 8;       // ring slots
     static constexpr int kQOff = 0;
-    static constexpr int kKOff = kQOff + kQBytes;
-    static constexpr int kVOff = kKOff + kStages * kKVBytes;
-    static constexpr int kBarOff = kVOff + kStages * kKVBytes;
-    static constexpr int kTotal = kBarOff + 128;
-    static constexpr int kDynamic = kTotal + 1024;         // slack for manual 1024-byte alignment
-    static constexpr int kTmemCols = (D == 128) ? 256 : 128;
-    static constexpr int kColS = 0;                        // S: 64 fp32 columns; P (bf16) reuses 0..31
-    static constexpr int kColO = 64;                       // O: D fp32 columns
+    static constexpr int kRingOff = kQBytes;
+    static constexpr int kBarOff = kRingOff + kRing * kTileBytes;
+    static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1;
+    static constexpr int kMiscOff = kBarOff + 8 * kNumBars;
+    static constexpr int kTotal = kMiscOff + 16;
+    static constexpr int kTmemCols = 256;
+    static constexpr int kColS = 0;                        // S buffers: 2 x 64 fp32 columns
+    static constexpr int kColO = 128;                      // O: D fp32 columns
 };
 
+struct Unit {
+    int seq0, j, cnt, rows_valid, kvh, tok0;
+    const int32_t* list;
+};
+
+// Unit u of the hand-out order -> what to compute.  KV-head-major, so that the K/V of one
+// head stay hot in L2 while its query blocks are processed; inside a head longest list first.
+__device__ __forceinline__ void decode_unit(const AttnArgs& a, int nqb, int u, Unit& un) {
+    const int idx = u % nqb;
+    un.kvh = u / nqb;
+    int seq, slot;
+    if (!a.dense) {
+        slot = a.order ? a.order[idx] : idx;
+        seq = a.qb_seq[slot];
+        un.j = a.qb_block[slot];
+        int c = a.kv_count[slot];
+        un.cnt = min(max(c, 1), a.max_degree);
+        un.list = a.kv_idx + (size_t)slot * a.max_degree;
+    } else {
+        slot = nqb - 1 - idx;
+        int acc = 0;
+        seq = 0;
+        un.j = 0;
+        for (int s = 0; s < a.batch; ++s) {
+            const int nb = (a.cu_seqlens[s + 1] - a.cu_seqlens[s] + kBlock - 1) / kBlock;
+            if (slot < acc + nb) { seq = s; un.j = slot - acc; break; }
+            acc += nb;
+        }
+        un.cnt = un.j + 1;
+        un.list = nullptr;
+    }
+    un.seq0 = a.cu_seqlens[seq];
+    const int seqlen = a.cu_seqlens[seq + 1] - un.seq0;
+    un.rows_valid = min(kBlock, seqlen - un.j * kBlock);
+    un.tok0 = un.seq0 + un.j * kBlock;
+}
+
 template <int D>
-__global__ void __launch_bounds__(kThreads) attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q,
-                                                            const __grid_constant__ CUtensorMap tm_k,
-                                                            const __grid_constant__ CUtensorMap tm_v,
-                                                            const AttnArgs args) {
-    using L = Smem<D>;
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
+__global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                               const __grid_constant__ CUtensorMap tm_k,
+                                                               const __grid_constant__ CUtensorMap tm_v,
+                                                               const AttnArgs args) {
+    using C = Cfg<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
 
-    // ---- which unit --------------------------------------------------------------------
-    const int slot = blockIdx.x;
-    const int kvh = blockIdx.y;
-    int seq, j, cnt;
-    const int32_t* list = nullptr;
-    if (args.status && (*args.status & BF1_DEV_WAIT_TIMEOUT)) return;
-    if (!args.dense) {
-        if (slot >= *args.num_qblocks) return;
-        seq = args.qb_seq[slot];
-        j = args.qb_block[slot];
-        cnt = args.kv_count[slot];
-        list = args.kv_idx + (size_t)slot * args.max_degree;
-    } else {
-        int acc = 0;
-        seq = -1;
-        j = 0;
-        for (int s = 0; s < args.batch; ++s) {
-            const int nb = (args.cu_seqlens[s + 1] - args.cu_seqlens[s] + kBlock - 1) / kBlock;
-            if (slot < acc + nb) { seq = s; j = slot - acc; break; }
-            acc += nb;
-        }
-        if (seq < 0) return;
-        cnt = j + 1;
-    }
-    const int seq0 = args.cu_seqlens[seq];
-    const int seqlen = args.cu_seqlens[seq + 1] - seq0;
-    const int rows_valid = min(kBlock, seqlen - j * kBlock);
-    const int tok0 = seq0 + j * kBlock;   // first token row of the query block
+    if (args.status && (*args.status & BF1_DEV_WAIT_TIMEOUT)) return;   // an earlier launch gave up
 
-    // ---- shared memory carve-up ----------------------------------------------------------
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = base + L::kQOff;
-    const uint32_t sK = base + L::kKOff;
-    const uint32_t sV = base + L::kVOff;
-    const uint32_t bar_q = base + L::kBarOff;
-    const uint32_t bar_kv = bar_q + 8;            // [kStages]
-    const uint32_t bar_s = bar_kv + 8 * kStages;
-    const uint32_t bar_o = bar_s + 8;
+    const uint32_t base = smem_u32(smem);
+    const uint32_t sQ = base + C::kQOff;
+    const uint32_t sRing = base + C::kRingOff;
+    const uint32_t bar_q_full = base + C::kBarOff;
+    const uint32_t bar_q_free = bar_q_full + 8;
+    const uint32_t bar_full = bar_q_free + 8;                 // [kRing]
+    const uint32_t bar_free = bar_full + 8 * C::kRing;        // [kRing]
+    const uint32_t bar_s_full = bar_free + 8 * C::kRing;      // [2]
+    const uint32_t bar_p_full = bar_s_full + 16;              // [2]
+    const uint32_t bar_pv_done = bar_p_full + 16;             // [2]
+    const uint32_t bar_o_free = bar_pv_done + 16;
+    uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + C::kMiscOff);
+    int* s_abort = reinterpret_cast<int*>(smem + C::kMiscOff + 4);
+    int* s_nqb = reinterpret_cast<int*>(smem + C::kMiscOff + 8);
 
     if (tid == 0) {
-        s_abort = 0;
-        mbar_init(bar_q, 1);
-        for (int s = 0; s < kStages; ++s) mbar_init(bar_kv + 8 * s, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        *s_abort = 0;
+        if (base & 1023u) {   // the swizzled tiles need a 1024-byte aligned window
+            *s_abort = 1;
+            if (args.status) atomicOr(args.status, BF1_DEV_WAIT_TIMEOUT);
+        }
+        int nqb = 0;
+        if (!args.dense) {
+            nqb = min(*args.num_qblocks, args.capacity);
+        } else {
+            for (int s = 0; s < args.batch; ++s)
+                nqb += (args.cu_seqlens[s + 1] - args.cu_seqlens[s] + kBlock - 1) / kBlock;
+        }
+        *s_nqb = nqb;
+        mbar_init(bar_q_full, 1);
+        mbar_init(bar_q_free, 1);
+        for (int s = 0; s < C::kRing; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_free + 8 * s, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_s_full + 8 * s, 1);
+            mbar_init(bar_p_full + 8 * s, 4);    // one arrival per softmax warp
+            mbar_init(bar_pv_done + 8 * s, 1);
+        }
+        mbar_init(bar_o_free, 4);
         fence_mbar_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
     }
     __syncwarp();
-    if (warp == 0) {
-        tmem_alloc(smem_u32(&s_tmem_base), L::kTmemCols);
+    if (warp == 1) {
+        tmem_alloc(smem_u32(s_tmem_base), C::kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = s_tmem_base;
-    const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);  // this warp's 32 lanes
-    volatile int* abort_flag = &s_abort;
+    const uint32_t tmem = *s_tmem_base;
+    volatile int* abort_flag = s_abort;
+    const int nqb = *s_nqb;
+    const int total_units = nqb * args.hkv;
 
-    // row of this thread: head (tid / 64) of the pair, token (tid % 64) of the block
-    const int hl = tid >> 6;
-    const int tl = tid & 63;
-
-    auto issue_kv = [&](int it) {
-        int p = args.dense ? it : list[it];
-        if (p < 0 || p > j || (it == cnt - 1) != (p == j)) {   // never index outside the sequence
-            if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
-            p = (it == cnt - 1) ? j : 0;
-        }
-        const int st = it % kStages;
-        const uint32_t bar = bar_kv + 8 * st;
-        mbar_expect_tx(bar, 2 * L::kKVBytes);
-        const int row = seq0 + p * kBlock;
+    if (warp == 0) {
+        // ================================ TMA producer ====================================
+        if (lane == 0) {
+            int slot = 0, pass = 0, n = 0;
+            for (int u = blockIdx.x; u < total_units && !*abort_flag; u += gridDim.x, ++n) {
+                Unit un;
+                decode_unit(args, nqb, u, un);
+                if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
+                mbar_expect_tx(bar_q_full, C::kQBytes);
 #pragma unroll
-        for (int c = 0; c < L::kChunks; ++c) {
-            tma_load_3d(sK + st * L::kKVBytes + c * (kBlock * 128), &tm_k, c * 64, kvh, row, bar);
-            tma_load_3d(sV + st * L::kKVBytes + c * (kBlock * 128), &tm_v, c * 64, kvh, row, bar);
-        }
-    };
-
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, L::kQBytes);
+                for (int c = 0; c < C::kChunks; ++c)
 #pragma unroll
-        for (int c = 0; c < L::kChunks; ++c)
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_3d(sQ + c * (kRows * 128) + h * (kBlock * 128), &tm_q, c * 64, un.kvh * 2 + h,
+                                    un.tok0, bar_q_full);
+                auto load_tile = [&](int i, bool is_v) {
+                    int p = args.dense ? i : un.list[i];
+                    if (p < 0 || p > un.j || (i == un.cnt - 1) != (p == un.j)) {   // stay inside the sequence
+                        if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
+                        p = (i == un.cnt - 1) ? un.j : 0;
+                    }
+                    if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
+                    const uint32_t bar = bar_full + 8 * slot;
+                    mbar_expect_tx(bar, C::kTileBytes);
+                    const uint32_t dst = sRing + slot * C::kTileBytes;
+                    const int row = un.seq0 + p * kBlock;
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
-                tma_load_3d(sQ + c * (kRows * 128) + h * (kBlock * 128), &tm_q, c * 64, kvh * 2 + h, tok0, bar_q);
-        issue_kv(0);
-    }
-    __syncwarp();
-
-    constexpr uint32_t kIdescS = idesc_bf16_f32(kBlock, false);   // 128 x 64 x 16, K-major B
-    constexpr uint32_t kIdescO = idesc_bf16_f32(D, true);         // 128 x D x 16, MN-major B
-
-    float m_run = -INFINITY;   // running maximum of the raw (unscaled) scores
-    float l_run = 0.f;         // running sum of exp2(scaled score - scaled max)
-
-    for (int it = 0; it < cnt; ++it) {
-        const int st = it % kStages;
-        const bool diag = (it == cnt - 1);
-        if (tid == 0) {
-            if (it + 1 < cnt) issue_kv(it + 1);   // stage (it+1)%2 was released by bar_o of it-1
-            if (it == 0) mbar_wait(bar_q, 0, abort_flag, args.status);
-            mbar_wait(bar_kv + 8 * st, (it / kStages) & 1, abort_flag, args.status);
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t a = sQ + (kk / 4) * (kRows * 128) + (kk % 4) * 32;
-                const uint32_t b = sK + st * L::kKVBytes + (kk / 4) * (kBlock * 128) + (kk % 4) * 32;
-                mma_ss(tmem + L::kColS, smem_desc_sw128(a, 16, 1024), smem_desc_sw128(b, 16, 1024), kIdescS,
-                       kk > 0);
+                    for (int c = 0; c < C::kChunks; ++c)
+                        tma_load_3d(dst + c * (kBlock * 128), is_v ? &tm_v : &tm_k, c * 64, un.kvh, row, bar);
+                    if (++slot == C::kRing) { slot = 0; ++pass; }
+                };
+                load_tile(0, false);
+                for (int i = 1; i < un.cnt; ++i) {
+                    load_tile(i, false);
+                    load_tile(i - 1, true);
+                }
+                load_tile(un.cnt - 1, true);
             }
-            mma_commit(bar_s);
         }
         __syncwarp();
-        mbar_wait(bar_s, it & 1, abort_flag, args.status);
-        tc_fence_after();
-
-        // ---- softmax on this thread's row ----------------------------------------------
-        uint32_t sreg[2][32];
-        tmem_ld32(t_lane + L::kColS, sreg[0]);
-        tmem_ld32(t_lane + L::kColS + 32, sreg[1]);
-        tmem_wait_ld();
-        float mx = m_run;
+    } else if (warp == 1) {
+        // ================================ MMA issuer ======================================
+        if (lane == 0) {
+            constexpr uint32_t kIdescS = idesc_bf16_f32(kBlock, false);   // 128 x 64 x 16, K-major B
+            constexpr uint32_t kIdescO = idesc_bf16_f32(D, true);         // 128 x D x 16, MN-major B
+            int slot = 0, pass = 0, n = 0;
+            uint32_t g = 0;   // tiles issued so far by this CTA; S buffer = g & 1
+            auto issue_s = [&](uint32_t gt) {
+                mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);
+                tc_fence_after();
+                const uint32_t kbase = sRing + slot * C::kTileBytes;
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t a = sQ + (kk / 4) * (kRows * 128) + (kk % 4) * 32;
+                    const uint32_t b = kbase + (kk / 4) * (kBlock * 128) + (kk % 4) * 32;
+                    mma_ss(tmem + C::kColS + (gt & 1) * 64, smem_desc_sw128(a, 16, 1024),
+                           smem_desc_sw128(b, 16, 1024), kIdescS, kk > 0);
+                }
+                mma_commit(bar_free + 8 * slot);
+                mma_commit(bar_s_full + 8 * (gt & 1));
+                if (++slot == C::kRing) { slot = 0; ++pass; }
+            };
+            for (int u = blockIdx.x; u < total_units && !*abort_flag; u += gridDim.x, ++n) {
+                Unit un;
+                decode_unit(args, nqb, u, un);
+                mbar_wait(bar_q_full, n & 1, abort_flag, args.status);
+                issue_s(g);
+                if (un.cnt == 1) mma_commit(bar_q_free);
+                for (int i = 0; i < un.cnt; ++i, ++g) {
+                    if (i + 1 < un.cnt) {
+                        issue_s(g + 1);
+                        if (i + 2 == un.cnt) mma_commit(bar_q_free);   // last S of the unit: Q may be replaced
+                    }
+                    mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);           // V(i) landed
+                    mbar_wait(bar_p_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);  // P(i) written
+                    if (i == 0 && n > 0) mbar_wait(bar_o_free, (n - 1) & 1, abort_flag, args.status);
+                    tc_fence_after();
+                    const uint32_t vbase = sRing + slot * C::kTileBytes;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                float s = __uint_as_float(sreg[h][c]);
-                if (diag && (h * 32 + c > tl)) s = -INFINITY;   // causal triangle, self block only
-                sreg[h][c] = __float_as_uint(s);
-                mx = fmaxf(mx, s);
+                    for (int kk = 0; kk < kBlock / 16; ++kk) {
+                        // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
+                        // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
+                        mma_ts(tmem + C::kColO, tmem + C::kColS + (g & 1) * 64 + kk * 8,
+                               smem_desc_sw128(vbase + kk * 2048, kBlock * 128, 1024), kIdescO, (i > 0 || kk > 0));
+                    }
+                    mma_commit(bar_free + 8 * slot);
+                    mma_commit(bar_pv_done + 8 * (g & 1));
+                    if (++slot == C::kRing) { slot = 0; ++pass; }
+                }
             }
-        const float alpha = ex2_approx((m_run - mx) * args.scale_log2);
-        const float msc = mx * args.scale_log2;
-        float rowsum = 0.f;
-        uint32_t preg[32];
-#pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const int h = c >> 4, cc = (c & 15) * 2;
-            const float p0 = ex2_approx(fmaf(__uint_as_float(sreg[h][cc]), args.scale_log2, -msc));
-            const float p1 = ex2_approx(fmaf(__uint_as_float(sreg[h][cc + 1]), args.scale_log2, -msc));
-            rowsum += p0 + p1;
-            preg[c] = pack_bf16x2(p0, p1);
         }
-        l_run = l_run * alpha + rowsum;
-        m_run = mx;
-        tmem_st32(t_lane + L::kColS, preg);   // P overwrites the first 32 columns of S
-        if (it > 0) {                         // rescale the running output
+        __syncwarp();
+    } else {
+        // ================================ softmax + epilogue ===============================
+        const int quarter = warp & 3;                     // TMEM lanes this warp may touch
+        const int row = quarter * 32 + lane;              // tile row of this thread
+        const int hl = row >> 6;                          // which head of the pair
+        const int tl = row & 63;                          // token inside the query block
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        const float c2 = args.scale_log2;
+        uint32_t g = 0;
+        int n = 0;
+        for (int u = blockIdx.x; u < total_units && !*abort_flag; u += gridDim.x, ++n) {
+            Unit un;
+            decode_unit(args, nqb, u, un);
+            float m_used = 0.f;    // reference maximum (raw score units) the exponentials are taken against
+            float l_run = 0.f;     // running sum of exp2((s - m_used) * c2)
+            for (int i = 0; i < un.cnt; ++i, ++g) {
+                const uint32_t t_s = t_lane + C::kColS + (g & 1) * 64;
+                mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);
+                tc_fence_after();
+                uint32_t sreg[2][32];
+                tmem_ld32(t_s, sreg[0]);
+                tmem_ld32(t_s + 32, sreg[1]);
+                tmem_wait_ld();
+                const bool diag = (i == un.cnt - 1);
+                float mx = -INFINITY;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        float s = __uint_as_float(sreg[h][c]);
+                        if (diag && (h * 32 + c > tl)) s = -INFINITY;   // causal triangle, self block only
+                        sreg[h][c] = __float_as_uint(s);
+                        mx = fmaxf(mx, s);
+                    }
+                if (i == 0) {
+                    m_used = mx;
+                } else {
+                    const bool need = (mx - m_used) * c2 > kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, need)) {
+                        const float m_new = fmaxf(m_used, mx);
+                        const float alpha = ex2_approx((m_used - m_new) * c2);
+                        l_run *= alpha;
+                        m_used = m_new;
+                        // O holds the sum up to tile i-1 once PV(g-1) has completed
+                        mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t oreg[32];
+                            tmem_ld32(t_lane + C::kColO + c * 32, oreg);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
+                            tmem_st32(t_lane + C::kColO + c * 32, oreg);
+                        }
+                    }
+                }
+                const float msc = m_used * c2;
+                float rowsum = 0.f;
+                uint32_t preg[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const int h = c >> 4, cc = (c & 15) * 2;
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(sreg[h][cc]), c2, -msc));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(sreg[h][cc + 1]), c2, -msc));
+                    rowsum += p0 + p1;
+                    preg[c] = pack_bf16x2(p0, p1);
+                }
+                l_run += rowsum;
+                tmem_st32(t_s, preg);   // P overwrites the first 32 columns of this S buffer
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p_full + 8 * (g & 1));
+            }
+            // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------
+            mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
+            tc_fence_after();
+            const float inv_l = 1.f / l_run;
+            const int tok = un.tok0 + tl;
+            const bool store = tl < un.rows_valid;
+            __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (un.kvh * 2 + hl)) * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t oreg[32];
-                tmem_ld32(t_lane + L::kColO + c * 32, oreg);
+                tmem_ld32(t_lane + C::kColO + c * 32, oreg);
                 tmem_wait_ld();
+                if (c == D / 32 - 1) {   // O has been read out: the next unit may overwrite it
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_o_free);
+                }
+                if (store) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
-                tmem_st32(t_lane + L::kColO + c * 32, oreg);
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(oreg[e + 0]) * inv_l, __uint_as_float(oreg[e + 1]) * inv_l);
+                        w.y = pack_bf16x2(__uint_as_float(oreg[e + 2]) * inv_l, __uint_as_float(oreg[e + 3]) * inv_l);
+                        w.z = pack_bf16x2(__uint_as_float(oreg[e + 4]) * inv_l, __uint_as_float(oreg[e + 5]) * inv_l);
+                        w.w = pack_bf16x2(__uint_as_float(oreg[e + 6]) * inv_l, __uint_as_float(oreg[e + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + e) = w;
+                    }
+                }
+            }
+            if (store) {
+                const float lse2 = m_used * c2 + lg2_approx(l_run);   // log2 domain
+                args.lse[(size_t)(un.kvh * 2 + hl) * args.total_tokens + tok] = lse2 * 0.6931471805599453f;
             }
         }
-        tmem_wait_st();
-        tc_fence_before();
-        __syncthreads();
-
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < kBlock / 16; ++kk) {
-                // V tile: rows = kv tokens (K of this MMA), 128-byte rows of 64 d-elements;
-                // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
-                const uint32_t b = sV + st * L::kKVBytes + kk * 2048;
-                mma_ts(tmem + L::kColO, tmem + L::kColS + kk * 8, smem_desc_sw128(b, kBlock * 128, 1024),
-                       kIdescO, (it > 0 || kk > 0));
-            }
-            mma_commit(bar_o);
-        }
-        __syncwarp();
-        mbar_wait(bar_o, it & 1, abort_flag, args.status);
-        tc_fence_after();
-    }
-
-    // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
-    const float inv_l = 1.f / l_run;
-    const int tok = tok0 + tl;
-    const bool store = tl < rows_valid;
-    __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * 2 + hl)) * D;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-        uint32_t oreg[32];
-        tmem_ld32(t_lane + L::kColO + c * 32, oreg);
-        tmem_wait_ld();
-        if (store) {
-#pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-                uint4 w;
-                w.x = pack_bf16x2(__uint_as_float(oreg[e + 0]) * inv_l, __uint_as_float(oreg[e + 1]) * inv_l);
-                w.y = pack_bf16x2(__uint_as_float(oreg[e + 2]) * inv_l, __uint_as_float(oreg[e + 3]) * inv_l);
-                w.z = pack_bf16x2(__uint_as_float(oreg[e + 4]) * inv_l, __uint_as_float(oreg[e + 5]) * inv_l);
-                w.w = pack_bf16x2(__uint_as_float(oreg[e + 6]) * inv_l, __uint_as_float(oreg[e + 7]) * inv_l);
-                *reinterpret_cast<uint4*>(orow + c * 32 + e) = w;
-            }
-        }
-    }
-    if (store) {
-        const float lse2 = m_run * args.scale_log2 + lg2_approx(l_run);   // log2 domain
-        args.lse[(size_t)(kvh * 2 + hl) * args.total_tokens + tok] = lse2 * 0.6931471805599453f;
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, L::kTmemCols);
+    if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
 }
 
 // ---- host side ---------------------------------------------------------------------------
@@ -322,28 +424,30 @@ static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d) {
     return BF1_OK;
 }
 
-static int check_device() {
+struct DeviceInfo {
+    int sm_count = 0;
+    bool ok = false;
+};
+
+static int device_info(DeviceInfo* out) {
+    static DeviceInfo cache[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(BF1_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e));
-    int major = 0;
-    BF1_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
-    if (major != 10) return fail(BF1_ERR_NO_DEVICE, "device compute capability %d.x is not sm_100", major);
-    return BF1_OK;
-}
-
-template <int D>
-static int launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnArgs& a,
-                  int slots, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            Smem<D>::kDynamic));
-        configured = true;
+    if (dev < 0 || dev >= 64) return fail(BF1_ERR_NO_DEVICE, "device ordinal %d out of range", dev);
+    if (!cache[dev].ok) {
+        int major = 0, sms = 0;
+        BF1_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major != 10) return fail(BF1_ERR_NO_DEVICE, "device compute capability %d.x is not sm_100", major);
+        BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            Cfg<128>::kTotal));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            Cfg<64>::kTotal));
+        cache[dev].sm_count = sms;
+        cache[dev].ok = true;
     }
-    dim3 grid(slots, a.hkv);
-    attn_fwd_kernel<D><<<grid, kThreads, Smem<D>::kDynamic, stream>>>(tq, tk, tv, a);
-    BF1_CUDA_CHECK(cudaGetLastError());
+    *out = cache[dev];
     return BF1_OK;
 }
 
@@ -362,8 +466,7 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15)
         return fail(BF1_ERR_INVALID_ARG, "q, k, v and o must be 16-byte aligned");
-    if (hkv > 65535) return fail(BF1_ERR_UNSUPPORTED, "hkv %d exceeds the grid limit", hkv);
-    int slots;
+    int64_t slots;
     if (route) {
         if (!route->qb_seq || !route->qb_block || !route->kv_count || !route->kv_idx || !route->num_qblocks ||
             !route->status)
@@ -372,12 +475,12 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
             return fail(BF1_ERR_CAPACITY, "route capacity_qblocks and max_degree must be >= 1");
         slots = route->capacity_qblocks;
     } else {
-        const int64_t cap = total_tokens / kBlock + batch;
-        if (cap > 0x7fffffffLL) return fail(BF1_ERR_UNSUPPORTED, "too many query blocks");
-        slots = (int)cap;
+        slots = total_tokens / kBlock + batch;
     }
+    if (slots * hkv > 0x7fffffffLL) return fail(BF1_ERR_UNSUPPORTED, "too many work units");
     if (total_tokens == 0 || batch == 0) return BF1_OK;   // nothing to do
-    if (int rc = check_device()) return rc;
+    DeviceInfo info;
+    if (int rc = device_info(&info)) return rc;
 
     CUtensorMap tq, tk, tv;
     if (int rc = make_map(&tq, q, total_tokens, hq, d)) return rc;
@@ -397,13 +500,22 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     a.qb_block = route ? route->qb_block : nullptr;
     a.kv_count = route ? route->kv_count : nullptr;
     a.kv_idx = route ? route->kv_idx : nullptr;
+    a.order = route ? route->order : nullptr;
     a.num_qblocks = route ? route->num_qblocks : nullptr;
     a.max_degree = route ? route->max_degree : 0;
+    a.capacity = route ? route->capacity_qblocks : 0;
     a.status = route ? route->status : status_dev;
     a.o = reinterpret_cast<__nv_bfloat16*>(o);
     a.lse = lse;
-    if (d == 128) return launch<128>(tq, tk, tv, a, slots, (cudaStream_t)stream);
-    return launch<64>(tq, tk, tv, a, slots, (cudaStream_t)stream);
+
+    const int64_t units = slots * hkv;
+    const int grid = (int)(units < 2LL * info.sm_count ? units : 2LL * info.sm_count);
+    if (d == 128)
+        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
+    else
+        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
+    BF1_CUDA_CHECK(cudaGetLastError());
+    return BF1_OK;
 }
 
 }  // namespace bf1
