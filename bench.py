@@ -186,7 +186,8 @@ def sweep(bf1, dev):
         lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
         stream = torch.cuda.current_stream()
         f_s = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
-        f_d = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse)
+        work = torch.zeros(4, dtype=torch.int32, device=dev)
+        f_d = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse, work=work)
         meds = {"bf1": [], "dense": []}
         for order in (("dense", "bf1"), ("bf1", "dense")):
             for which in order:
@@ -217,8 +218,9 @@ def run_single(args):
     o = torch.empty_like(q)
     lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
+    work = torch.zeros(4, dtype=torch.int32, device=dev)
     if args.mode == "dense":
-        f = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse)
+        f = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse, work=work)
         pairs = sum(n * (n + 1) // 2 for n in w.seqlens)
     else:
         f = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)

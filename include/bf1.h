@@ -89,6 +89,11 @@ typedef struct {
     int32_t *num_qblocks;      /* [1] slots actually used                                 */
     int32_t *status;           /* [1] BF1_DEV_* bits; 0 = fine.  Written (not OR-ed) by
                                   bf1_plan_route, OR-ed by the attention entry points     */
+    int32_t *sched;            /* [2] work hand-out counters of the attention kernel: zeroed
+                                  by bf1_plan_route and put back to zero by every
+                                  bf1_attn_fwd launch when it finishes.  Launches that share
+                                  a route must therefore be ordered (same stream, or
+                                  otherwise not overlapping on the GPU)                    */
 } bf1_route;
 
 /* Host-only helper: how large the route arrays must be for a batch of `batch` sequences,
@@ -126,12 +131,15 @@ int bf1_attn_fwd(const void *q, const void *k, const void *v, const int32_t *cu_
 
 /* Dense causal attention through the same kernel (every predecessor block selected):
  * the paper's dense comparator (Section 4.3) and its dense-path equivalence gate
- * (Section 4.2).  Arguments as bf1_attn_fwd without the route; `status_dev` is an optional
- * [1] int32 device word for BF1_DEV_* bits (may be NULL). */
+ * (Section 4.2).  Arguments as bf1_attn_fwd without the route.  `work_dev` is an optional
+ * [4] int32 device array, all zero before its first use: word 0 receives BF1_DEV_* bits,
+ * words 1..2 are the work hand-out counters (left at zero by every launch; launches sharing
+ * the array must be ordered), word 3 is reserved.  NULL selects a static work split and
+ * drops device-side error reporting. */
 int bf1_dense_causal_fwd(const void *q, const void *k, const void *v,
                          const int32_t *cu_seqlens_dev, int32_t batch, int64_t total_tokens,
                          int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d,
-                         float softmax_scale, void *o, float *lse, int32_t *status_dev,
+                         float softmax_scale, void *o, float *lse, int32_t *work_dev,
                          void *stream);
 
 /* Message for the last non-OK status returned on the calling thread ("" if none). */

@@ -38,7 +38,7 @@ class _RouteC(ctypes.Structure):
                 ("kv_count", ctypes.c_void_p), ("kv_idx", ctypes.c_void_p),
                 ("pair_count", ctypes.c_void_p), ("order", ctypes.c_void_p),
                 ("total_pairs", ctypes.c_void_p), ("num_qblocks", ctypes.c_void_p),
-                ("status", ctypes.c_void_p)]
+                ("status", ctypes.c_void_p), ("sched", ctypes.c_void_p)]
 
 
 class Bf1Error(RuntimeError):
@@ -107,6 +107,7 @@ class Route:
     total_pairs: torch.Tensor
     num_qblocks: torch.Tensor
     status: torch.Tensor
+    sched: torch.Tensor
     c: _RouteC = None
 
     @staticmethod
@@ -118,10 +119,12 @@ class Route:
                   kv_idx=torch.empty((capacity_qblocks, max_degree), **i32),
                   pair_count=torch.empty(capacity_qblocks, **i32), order=torch.empty(capacity_qblocks, **i32),
                   total_pairs=torch.zeros(1, dtype=torch.int64, device=device),
-                  num_qblocks=torch.zeros(1, **i32), status=torch.zeros(1, **i32))
+                  num_qblocks=torch.zeros(1, **i32), status=torch.zeros(1, **i32),
+                  sched=torch.zeros(2, **i32))
         r.c = _RouteC(capacity_qblocks, max_degree, r.qb_seq.data_ptr(), r.qb_block.data_ptr(),
                       r.kv_count.data_ptr(), r.kv_idx.data_ptr(), r.pair_count.data_ptr(), r.order.data_ptr(),
-                      r.total_pairs.data_ptr(), r.num_qblocks.data_ptr(), r.status.data_ptr())
+                      r.total_pairs.data_ptr(), r.num_qblocks.data_ptr(), r.status.data_ptr(),
+                      r.sched.data_ptr())
         return r
 
     def check_status(self):
@@ -173,8 +176,9 @@ def attn_fwd(q, k, v, cu_seqlens, max_seqlen: int, route: Route, scale: Optional
 
 
 def dense_causal_fwd(q, k, v, cu_seqlens, max_seqlen: int, scale: Optional[float] = None, out=None,
-                     lse=None, status=None, stream=None):
-    """bf1_dense_causal_fwd: plain causal attention through the same kernel."""
+                     lse=None, work=None, stream=None):
+    """bf1_dense_causal_fwd: plain causal attention through the same kernel.  `work`: optional
+    zero-initialised int32[4] CUDA tensor (word 0 = device status, words 1..2 = hand-out counters)."""
     T, hq, hkv, d = _check_qkv(q, k, v)
     if out is None:
         out = torch.empty_like(q)
@@ -183,7 +187,7 @@ def dense_causal_fwd(q, k, v, cu_seqlens, max_seqlen: int, scale: Optional[float
     _check(load().bf1_dense_causal_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), cu_seqlens.data_ptr(),
                                        cu_seqlens.numel() - 1, T, max_seqlen, hq, hkv, d,
                                        float(scale) if scale else 0.0, out.data_ptr(), lse.data_ptr(),
-                                       status.data_ptr() if status is not None else None,
+                                       work.data_ptr() if work is not None else None,
                                        _stream_ptr(stream)))
     return out, lse
 

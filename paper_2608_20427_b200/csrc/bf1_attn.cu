@@ -50,6 +50,7 @@ struct AttnArgs {
     int32_t max_degree;
     int32_t capacity;
     int32_t* status;       // may be null in dense mode
+    int32_t* sched;        // [2] dynamic hand-out counter + finished-CTA counter; null: static stride
     __nv_bfloat16* o;
     float* lse;
 };
@@ -63,9 +64,10 @@ struct Cfg {
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = kQBytes;
     static constexpr int kBarOff = kRingOff + kRing * kTileBytes;
-    static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1;
+    static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1 + 2;
     static constexpr int kMiscOff = kBarOff + 8 * kNumBars;
-    static constexpr int kTotal = kMiscOff + 16;
+    static constexpr int kInfoOff = kMiscOff + 16;             // two int4 unit descriptors
+    static constexpr int kTotal = kInfoOff + 32;
     static constexpr int kTmemCols = 256;
     static constexpr int kColS = 0;                        // S buffers: 2 x 64 fp32 columns
     static constexpr int kColO = 128;                      // O: D fp32 columns
@@ -120,7 +122,22 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const int warp = tid >> 5;
     const int lane = tid & 31;
 
-    if (args.status && (*args.status & BF1_DEV_WAIT_TIMEOUT)) return;   // an earlier launch gave up
+    // Dynamic hand-out: sched[0] is the next unit, sched[1] counts CTAs that are done; the last
+    // one to finish puts both back to zero, so the words are ready for the next launch.
+    auto retire = [&]() {
+        if (args.sched && threadIdx.x == 0) {
+            __threadfence();
+            if (atomicAdd(args.sched + 1, 1) == (int)gridDim.x - 1) {
+                args.sched[0] = 0;
+                args.sched[1] = 0;
+                __threadfence();
+            }
+        }
+    };
+    if (args.status && (*args.status & BF1_DEV_WAIT_TIMEOUT)) {   // an earlier launch gave up
+        retire();
+        return;
+    }
 
     const uint32_t base = smem_u32(smem);
     const uint32_t sQ = base + C::kQOff;
@@ -133,6 +150,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const uint32_t bar_p_full = bar_s_full + 16;              // [2]
     const uint32_t bar_pv_done = bar_p_full + 16;             // [2]
     const uint32_t bar_o_free = bar_pv_done + 16;
+    const uint32_t bar_info = bar_o_free + 8;                 // [2]
+    volatile int4* s_info = reinterpret_cast<volatile int4*>(smem + C::kInfoOff);   // {cnt, rows_valid, tok0, kvh}
     uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + C::kMiscOff);
     int* s_abort = reinterpret_cast<int*>(smem + C::kMiscOff + 4);
     int* s_nqb = reinterpret_cast<int*>(smem + C::kMiscOff + 8);
@@ -163,6 +182,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             mbar_init(bar_pv_done + 8 * s, 1);
         }
         mbar_init(bar_o_free, 4);
+        mbar_init(bar_info, 1);
+        mbar_init(bar_info + 8, 1);
         fence_mbar_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
@@ -184,11 +205,30 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     if (warp == 0) {
         // ================================ TMA producer ====================================
         if (lane == 0) {
-            int slot = 0, pass = 0, n = 0;
-            for (int u = blockIdx.x; u < total_units && !*abort_flag; u += gridDim.x, ++n) {
-                Unit un;
-                decode_unit(args, nqb, u, un);
+            int slot = 0, pass = 0;
+            auto next_unit = [&](int n) -> int {
+                return args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
+            };
+            Unit un = {};
+            bool have = false;
+            {
+                const int u = next_unit(0);
+                have = u < total_units;
+                if (have) decode_unit(args, nqb, u, un);
+            }
+            for (int n = 0;; ++n) {
                 if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
+                if (*abort_flag) have = false;
+                // publish the unit (or the end marker cnt = 0) to the other roles
+                s_info[n & 1].x = have ? un.cnt : 0;
+                s_info[n & 1].y = un.rows_valid;
+                s_info[n & 1].z = un.tok0;
+                s_info[n & 1].w = un.kvh;
+                mbar_arrive(bar_info + 8 * (n & 1));
+                if (!have) {
+                    mbar_arrive(bar_q_full);
+                    break;
+                }
                 mbar_expect_tx(bar_q_full, C::kQBytes);
 #pragma unroll
                 for (int c = 0; c < C::kChunks; ++c)
@@ -196,12 +236,15 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     for (int h = 0; h < 2; ++h)
                         tma_load_3d(sQ + c * (kRows * 128) + h * (kBlock * 128), &tm_q, c * 64, un.kvh * 2 + h,
                                     un.tok0, bar_q_full);
-                auto load_tile = [&](int i, bool is_v) {
+                auto entry = [&](int i) -> int {
                     int p = args.dense ? i : un.list[i];
                     if (p < 0 || p > un.j || (i == un.cnt - 1) != (p == un.j)) {   // stay inside the sequence
                         if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
                         p = (i == un.cnt - 1) ? un.j : 0;
                     }
+                    return p;
+                };
+                auto load_tile = [&](int p, bool is_v) {
                     if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
                     const uint32_t bar = bar_full + 8 * slot;
                     mbar_expect_tx(bar, C::kTileBytes);
@@ -212,12 +255,23 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                         tma_load_3d(dst + c * (kBlock * 128), is_v ? &tm_v : &tm_k, c * 64, un.kvh, row, bar);
                     if (++slot == C::kRing) { slot = 0; ++pass; }
                 };
-                load_tile(0, false);
+                // K0, K1, V0, K2, V1, ...: the order in which the MMA warp consumes them; list
+                // entries are fetched one tile ahead so that their latency hides behind the ring waits
+                int p_prev = entry(0);
+                int p_cur = un.cnt > 1 ? entry(1) : 0;
+                load_tile(p_prev, false);
                 for (int i = 1; i < un.cnt; ++i) {
-                    load_tile(i, false);
-                    load_tile(i - 1, true);
+                    const int p_next = (i + 1 < un.cnt) ? entry(i + 1) : 0;
+                    load_tile(p_cur, false);
+                    load_tile(p_prev, true);
+                    p_prev = p_cur;
+                    p_cur = p_next;
                 }
-                load_tile(un.cnt - 1, true);
+                load_tile(p_prev, true);
+                // decode the next unit now: the loads overlap the wait for the Q buffer
+                const int u = next_unit(n + 1);
+                have = u < total_units;
+                if (have) decode_unit(args, nqb, u, un);
             }
         }
         __syncwarp();
@@ -243,16 +297,16 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 mma_commit(bar_s_full + 8 * (gt & 1));
                 if (++slot == C::kRing) { slot = 0; ++pass; }
             };
-            for (int u = blockIdx.x; u < total_units && !*abort_flag; u += gridDim.x, ++n) {
-                Unit un;
-                decode_unit(args, nqb, u, un);
+            for (;; ++n) {
                 mbar_wait(bar_q_full, n & 1, abort_flag, args.status);
+                const int cnt = s_info[n & 1].x;
+                if (cnt == 0 || *abort_flag) break;
                 issue_s(g);
-                if (un.cnt == 1) mma_commit(bar_q_free);
-                for (int i = 0; i < un.cnt; ++i, ++g) {
-                    if (i + 1 < un.cnt) {
+                if (cnt == 1) mma_commit(bar_q_free);
+                for (int i = 0; i < cnt; ++i, ++g) {
+                    if (i + 1 < cnt) {
                         issue_s(g + 1);
-                        if (i + 2 == un.cnt) mma_commit(bar_q_free);   // last S of the unit: Q may be replaced
+                        if (i + 2 == cnt) mma_commit(bar_q_free);   // last S of the unit: Q may be replaced
                     }
                     mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);           // V(i) landed
                     mbar_wait(bar_p_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);  // P(i) written
@@ -283,30 +337,40 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         const float c2 = args.scale_log2;
         uint32_t g = 0;
         int n = 0;
-        for (int u = blockIdx.x; u < total_units && !*abort_flag; u += gridDim.x, ++n) {
+        for (;; ++n) {
+            mbar_wait(bar_info + 8 * (n & 1), (n >> 1) & 1, abort_flag, args.status);
             Unit un;
-            decode_unit(args, nqb, u, un);
+            un.cnt = s_info[n & 1].x;
+            un.rows_valid = s_info[n & 1].y;
+            un.tok0 = s_info[n & 1].z;
+            un.kvh = s_info[n & 1].w;
+            if (un.cnt == 0 || *abort_flag) break;
             float m_used = 0.f;    // reference maximum (raw score units) the exponentials are taken against
             float l_run = 0.f;     // running sum of exp2((s - m_used) * c2)
             for (int i = 0; i < un.cnt; ++i, ++g) {
                 const uint32_t t_s = t_lane + C::kColS + (g & 1) * 64;
                 mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);
                 tc_fence_after();
-                uint32_t sreg[2][32];
-                tmem_ld32(t_s, sreg[0]);
-                tmem_ld32(t_s + 32, sreg[1]);
+                uint32_t sreg[64];
+                {
+                    uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sreg[0]);
+                    uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sreg[32]);
+                    tmem_ld32(t_s, lo);
+                    tmem_ld32(t_s + 32, hi);
+                }
                 tmem_wait_ld();
-                const bool diag = (i == un.cnt - 1);
-                float mx = -INFINITY;
+                if (i == un.cnt - 1) {   // self block: causal triangle (warp-uniform branch)
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
+                    for (int c = 0; c < 64; ++c)
+                        if (c > tl) sreg[c] = 0xff800000u;   // -inf
+                }
+                float mxa = -INFINITY, mxb = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        float s = __uint_as_float(sreg[h][c]);
-                        if (diag && (h * 32 + c > tl)) s = -INFINITY;   // causal triangle, self block only
-                        sreg[h][c] = __float_as_uint(s);
-                        mx = fmaxf(mx, s);
-                    }
+                for (int c = 0; c < 64; c += 4) {
+                    mxa = fmax3(mxa, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+                    mxb = fmax3(mxb, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+                }
+                const float mx = fmaxf(mxa, mxb);
                 if (i == 0) {
                     m_used = mx;
                 } else {
@@ -331,16 +395,21 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     }
                 }
                 const float msc = m_used * c2;
-                float rowsum = 0.f;
+                const uint64_t c2p = pack2(c2, c2), mscp = pack2(-msc, -msc);
+                uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
                 uint32_t preg[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
-                    const int h = c >> 4, cc = (c & 15) * 2;
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(sreg[h][cc]), c2, -msc));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(sreg[h][cc + 1]), c2, -msc));
-                    rowsum += p0 + p1;
+                    const uint64_t x = fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2p, mscp);
+                    float x0, x1;
+                    unpack2(x, x0, x1);
+                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                    if (c & 1) sum_b = add2(sum_b, pack2(p0, p1)); else sum_a = add2(sum_a, pack2(p0, p1));
                     preg[c] = pack_bf16x2(p0, p1);
                 }
+                float r0, r1;
+                unpack2(add2(sum_a, sum_b), r0, r1);
+                const float rowsum = r0 + r1;
                 l_run += rowsum;
                 tmem_st32(t_s, preg);   // P overwrites the first 32 columns of this S buffer
                 tmem_wait_st();
@@ -387,6 +456,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
+    retire();
 }
 
 // ---- host side ---------------------------------------------------------------------------
@@ -453,7 +523,7 @@ static int device_info(DeviceInfo* out) {
 
 static int attn_common(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_dev, int32_t batch,
                        int64_t total_tokens, int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d,
-                       float softmax_scale, const bf1_route* route, void* o, float* lse, int32_t* status_dev,
+                       float softmax_scale, const bf1_route* route, void* o, float* lse, int32_t* work_dev,
                        void* stream) {
     if (!q || !k || !v || !o || !lse || !cu_seqlens_dev)
         return fail(BF1_ERR_INVALID_ARG, "a tensor pointer is null");
@@ -504,7 +574,8 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     a.num_qblocks = route ? route->num_qblocks : nullptr;
     a.max_degree = route ? route->max_degree : 0;
     a.capacity = route ? route->capacity_qblocks : 0;
-    a.status = route ? route->status : status_dev;
+    a.status = route ? route->status : work_dev;
+    a.sched = route ? route->sched : (work_dev ? work_dev + 1 : nullptr);
     a.o = reinterpret_cast<__nv_bfloat16*>(o);
     a.lse = lse;
 
@@ -532,7 +603,7 @@ extern "C" int bf1_attn_fwd(const void* q, const void* k, const void* v, const i
 extern "C" int bf1_dense_causal_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_dev,
                                     int32_t batch, int64_t total_tokens, int32_t max_seqlen, int32_t hq,
                                     int32_t hkv, int32_t d, float softmax_scale, void* o, float* lse,
-                                    int32_t* status_dev, void* stream) {
+                                    int32_t* work_dev, void* stream) {
     return bf1::attn_common(q, k, v, cu_seqlens_dev, batch, total_tokens, max_seqlen, hq, hkv, d, softmax_scale,
-                            nullptr, o, lse, status_dev, stream);
+                            nullptr, o, lse, work_dev, stream);
 }

@@ -34,16 +34,17 @@ def run_gpu(w, q, k, v, dense=False, scale=None, guard=0):
     out = poison((T + guard, w.hq, w.d), torch.bfloat16, dev)
     lse = poison((w.hq, T), torch.float32, dev)
     if dense:
-        status = torch.zeros(1, dtype=torch.int32, device=dev)
-        bf1.dense_causal_fwd(qd, kd, vd, cu, w.max_seqlen, scale=scale, out=out[:T], lse=lse, status=status)
+        work = torch.zeros(4, dtype=torch.int32, device=dev)
+        bf1.dense_causal_fwd(qd, kd, vd, cu, w.max_seqlen, scale=scale, out=out[:T], lse=lse, work=work)
         torch.cuda.synchronize()
-        assert int(status.item()) == 0
+        assert work.tolist() == [0, 0, 0, 0]
         route = None
     else:
         route = bf1.plan_route(cu, w.max_seqlen, lib_cfg(w))
         bf1.attn_fwd(qd, kd, vd, cu, w.max_seqlen, route, scale=scale, out=out[:T], lse=lse)
         torch.cuda.synchronize()
         route.check_status()
+        assert route.sched.tolist() == [0, 0]   # hand-out counters are back at zero
     if guard:
         assert torch.isnan(out[T:].float()).all(), "kernel wrote past the last token row"
     return out[:T].float().cpu().numpy(), lse.cpu().numpy(), route
