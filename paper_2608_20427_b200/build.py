@@ -27,13 +27,18 @@ def is_stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; return its path."""
-    if not force and not is_stale():
+def build(force: bool = False, verbose: bool = False, out: str = None, defines=()) -> str:
+    """Compile the library if it is missing or older than its sources; return its path.
+    `out` / `defines` build a variant (e.g. -DBF1_TRACE) somewhere else."""
+    if out is None and os.environ.get("BF1_LIB"):
+        return os.environ["BF1_LIB"]          # use a library built elsewhere (e.g. a trace build)
+    if out is None and not force and not is_stale():
         return LIB
-    tmp = LIB + ".tmp.%d" % os.getpid()
+    lib = out or LIB
+    tmp = lib + ".tmp.%d" % os.getpid()
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-o", tmp]
+    cmd += ["-D" + d for d in defines]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
@@ -42,8 +47,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         sys.stderr.write(res.stdout)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed building libbf1.so:\n" + res.stdout)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

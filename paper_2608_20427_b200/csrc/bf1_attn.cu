@@ -73,6 +73,35 @@ struct Cfg {
     static constexpr int kColO = 128;                      // O: D fp32 columns
 };
 
+// Optional event trace (compiled in with -DBF1_TRACE only): per traced CTA and role, a list of
+// (event code << 32 | index, clock64) pairs, for reading the pipeline's timeline off-line.
+#ifdef BF1_TRACE
+__device__ long long* g_trace_buf = nullptr;
+__device__ int g_trace_cap = 0;
+constexpr int kTraceCtas = 8;
+struct Tracer {
+    long long* p = nullptr;
+    int n = 0, cap = 0;
+    __device__ void init(int role) {
+        cap = g_trace_cap;
+        p = (g_trace_buf && blockIdx.x < kTraceCtas) ? g_trace_buf + ((size_t)(blockIdx.x * 3 + role)) * cap * 2 : nullptr;
+    }
+    __device__ void rec(int code, int idx) {
+        if (p && n < cap) {
+            p[2 * n] = ((long long)code << 32) | (unsigned)idx;
+            p[2 * n + 1] = clock64();
+            ++n;
+        }
+    }
+};
+#define TR(tr, code, idx) (tr).rec((code), (idx))
+#else
+struct Tracer {
+    __device__ void init(int) {}
+};
+#define TR(tr, code, idx) ((void)0)
+#endif
+
 struct Unit {
     int seq0, j, cnt, rows_valid, kvh, tok0;
     const int32_t* list;
@@ -206,6 +235,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         // ================================ TMA producer ====================================
         if (lane == 0) {
             int slot = 0, pass = 0;
+            Tracer tr;
+            tr.init(0);
+            int n_tiles = 0;
+            (void)n_tiles;
             auto next_unit = [&](int n) -> int {
                 return args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
             };
@@ -219,6 +252,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             for (int n = 0;; ++n) {
                 if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
                 if (*abort_flag) have = false;
+                TR(tr, 1, n);
                 // publish the unit (or the end marker cnt = 0) to the other roles
                 s_info[n & 1].x = have ? un.cnt : 0;
                 s_info[n & 1].y = un.rows_valid;
@@ -247,6 +281,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 auto load_tile = [&](int p, bool is_v) {
                     if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
                     const uint32_t bar = bar_full + 8 * slot;
+                    TR(tr, 2, n_tiles++);
                     mbar_expect_tx(bar, C::kTileBytes);
                     const uint32_t dst = sRing + slot * C::kTileBytes;
                     const int row = un.seq0 + p * kBlock;
@@ -272,56 +307,84 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 const int u = next_unit(n + 1);
                 have = u < total_units;
                 if (have) decode_unit(args, nqb, u, un);
+                TR(tr, 3, n);
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ================================ MMA issuer ======================================
-        if (lane == 0) {
+        // The whole warp walks the loop (so that addresses and descriptors stay warp-uniform and
+        // cheap); one elected lane issues the MMAs and commits.
+        {
             constexpr uint32_t kIdescS = idesc_bf16_f32(kBlock, false);   // 128 x 64 x 16, K-major B
             constexpr uint32_t kIdescO = idesc_bf16_f32(D, true);         // 128 x D x 16, MN-major B
             int slot = 0, pass = 0, n = 0;
             uint32_t g = 0;   // tiles issued so far by this CTA; S buffer = g & 1
+            Tracer tr;
+            if (lane == 0) tr.init(1);
+            // Descriptor halves that never change: the high word (SBO = 1024, version, swizzle) and
+            // the low words of Q's eight k-slices; a ring slot only adds slot * kTileBytes / 16.
+            constexpr uint32_t kDescHi = desc_hi_sw128(1024);
+            const uint32_t q_lo = desc_lo_sw128(sQ, 16);
+            const uint32_t k_lo0 = desc_lo_sw128(sRing, 16);
+            const uint32_t v_lo0 = desc_lo_sw128(sRing, kBlock * 128);
             auto issue_s = [&](uint32_t gt) {
+                TR(tr, 9, gt);
                 mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);
+                TR(tr, 10, gt);
                 tc_fence_after();
-                const uint32_t kbase = sRing + slot * C::kTileBytes;
+                const uint32_t k_lo = k_lo0 + slot * (C::kTileBytes >> 4);
+                const uint32_t d_s = tmem + C::kColS + (gt & 1) * 64;
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t a = sQ + (kk / 4) * (kRows * 128) + (kk % 4) * 32;
-                    const uint32_t b = kbase + (kk / 4) * (kBlock * 128) + (kk % 4) * 32;
-                    mma_ss(tmem + C::kColS + (gt & 1) * 64, smem_desc_sw128(a, 16, 1024),
-                           smem_desc_sw128(b, 16, 1024), kIdescS, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t a_off = ((kk / 4) * (kRows * 128) + (kk % 4) * 32) >> 4;
+                        const uint32_t b_off = ((kk / 4) * (kBlock * 128) + (kk % 4) * 32) >> 4;
+                        if (kk == 0) mma_ss_lohi<false>(d_s, q_lo + a_off, k_lo + b_off, kDescHi, kIdescS);
+                        else mma_ss_lohi<true>(d_s, q_lo + a_off, k_lo + b_off, kDescHi, kIdescS);
+                    }
+                    mma_commit(bar_free + 8 * slot);
+                    mma_commit(bar_s_full + 8 * (gt & 1));
                 }
-                mma_commit(bar_free + 8 * slot);
-                mma_commit(bar_s_full + 8 * (gt & 1));
+                __syncwarp();
                 if (++slot == C::kRing) { slot = 0; ++pass; }
             };
             for (;; ++n) {
                 mbar_wait(bar_q_full, n & 1, abort_flag, args.status);
                 const int cnt = s_info[n & 1].x;
+                TR(tr, 14, n);
                 if (cnt == 0 || *abort_flag) break;
                 issue_s(g);
-                if (cnt == 1) mma_commit(bar_q_free);
+                if (cnt == 1 && elect_one()) mma_commit(bar_q_free);
+                __syncwarp();
                 for (int i = 0; i < cnt; ++i, ++g) {
                     if (i + 1 < cnt) {
                         issue_s(g + 1);
-                        if (i + 2 == cnt) mma_commit(bar_q_free);   // last S of the unit: Q may be replaced
+                        // last S of the unit: Q may be replaced
+                        if (i + 2 == cnt && elect_one()) mma_commit(bar_q_free);
+                        __syncwarp();
                     }
                     mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);           // V(i) landed
+                    TR(tr, 11, g);
                     mbar_wait(bar_p_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);  // P(i) written
+                    TR(tr, 12, g);
                     if (i == 0 && n > 0) mbar_wait(bar_o_free, (n - 1) & 1, abort_flag, args.status);
+                    TR(tr, 13, g);
                     tc_fence_after();
-                    const uint32_t vbase = sRing + slot * C::kTileBytes;
+                    // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
+                    // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
+                    const uint32_t v_lo = v_lo0 + slot * (C::kTileBytes >> 4);
+                    const uint32_t a_p = tmem + C::kColS + (g & 1) * 64;
+                    if (elect_one()) {
+                        if (i == 0) mma_ts_lohi<false>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
+                        else mma_ts_lohi<true>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
 #pragma unroll
-                    for (int kk = 0; kk < kBlock / 16; ++kk) {
-                        // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
-                        // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
-                        mma_ts(tmem + C::kColO, tmem + C::kColS + (g & 1) * 64 + kk * 8,
-                               smem_desc_sw128(vbase + kk * 2048, kBlock * 128, 1024), kIdescO, (i > 0 || kk > 0));
+                        for (int kk = 1; kk < kBlock / 16; ++kk)
+                            mma_ts_lohi<true>(tmem + C::kColO, a_p + kk * 8, v_lo + kk * (2048 >> 4), kDescHi, kIdescO);
+                        mma_commit(bar_free + 8 * slot);
+                        mma_commit(bar_pv_done + 8 * (g & 1));
                     }
-                    mma_commit(bar_free + 8 * slot);
-                    mma_commit(bar_pv_done + 8 * (g & 1));
+                    __syncwarp();
                     if (++slot == C::kRing) { slot = 0; ++pass; }
                 }
             }
@@ -337,8 +400,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         const float c2 = args.scale_log2;
         uint32_t g = 0;
         int n = 0;
+        Tracer tr;
+        if (warp == 2 && lane == 0) tr.init(2);
         for (;; ++n) {
+            TR(tr, 23, n);
             mbar_wait(bar_info + 8 * (n & 1), (n >> 1) & 1, abort_flag, args.status);
+            TR(tr, 24, n);
             Unit un;
             un.cnt = s_info[n & 1].x;
             un.rows_valid = s_info[n & 1].y;
@@ -350,6 +417,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             for (int i = 0; i < un.cnt; ++i, ++g) {
                 const uint32_t t_s = t_lane + C::kColS + (g & 1) * 64;
                 mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);
+                TR(tr, 20, g);
                 tc_fence_after();
                 uint32_t sreg[64];
                 {
@@ -416,9 +484,11 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p_full + 8 * (g & 1));
+                TR(tr, 21, g);
             }
             // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------
             mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
+            TR(tr, 22, n);
             tc_fence_after();
             const float inv_l = 1.f / l_run;
             const int tok = un.tok0 + tl;
@@ -590,6 +660,14 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
 }
 
 }  // namespace bf1
+
+#ifdef BF1_TRACE
+extern "C" int bf1_trace_set(long long* buf_dev, int cap) {
+    cudaMemcpyToSymbol(bf1::g_trace_buf, &buf_dev, sizeof buf_dev);
+    cudaMemcpyToSymbol(bf1::g_trace_cap, &cap, sizeof cap);
+    return (int)cudaGetLastError();
+}
+#endif
 
 extern "C" int bf1_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_dev,
                             int32_t batch, int64_t total_tokens, int32_t max_seqlen, int32_t hq, int32_t hkv,
