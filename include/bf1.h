@@ -142,6 +142,30 @@ int bf1_dense_causal_fwd(const void *q, const void *k, const void *v,
                          float softmax_scale, void *o, float *lse, int32_t *work_dev,
                          void *stream);
 
+/* (The paper has no counterpart for this entry point; it exists for callers of this library.)
+ * BF1 forward for callers that cannot allocate device memory: code running after a server has
+ * fixed its memory budget, inside a real-time loop, or under an allocator that must not be
+ * re-entered.  It does what bf1_plan_route followed by bf1_attn_fwd do, but keeps the route
+ * arrays and the kernel's work hand-out counters in a fixed array inside the library (about
+ * 0.6 MB of device memory on every GPU that loads the library, held until the process exits),
+ * so the caller passes only inputs and outputs.
+ *   cfg         host; route parameters as for bf1_plan_route
+ *   status_dev  optional [1] int32 device word that receives the BF1_DEV_* bits (written by the
+ *               planner, OR-ed by the attention kernel); NULL keeps them inside the library
+ *   other arguments as bf1_attn_fwd
+ * Limits: the batch may hold at most 4096 query blocks (sum of ceil(n_s / 64); 262,144 tokens
+ * for lengths that are multiples of 64) and lists of at most 32 entries (the paper's route
+ * needs 3 + floor(log2(B-1))).  Beyond that the call returns BF1_ERR_CAPACITY and launches
+ * nothing.  It calls no cudaMalloc / cudaFree / allocating library routine.  The first call on a
+ * device looks up the array's address; make it before any stream capture.  All calls share the
+ * array and overwrite the previous call's contents, so calls that may overlap on the GPU
+ * (streams without ordering between them) race and must be avoided. */
+int bf1_attn_fwd_noalloc(const void *q, const void *k, const void *v, const int32_t *cu_seqlens_dev,
+                         int32_t batch, int64_t total_tokens, int32_t max_seqlen, int32_t hq,
+                         int32_t hkv, int32_t d, float softmax_scale,
+                         const bf1_route_cfg *cfg /* host */, void *o, float *lse,
+                         int32_t *status_dev, void *stream);
+
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char *bf1_last_error(void);
 

@@ -19,7 +19,7 @@ BF1_OK = 0
 DEV_BAD_SEQLENS, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_ROUTE = 1, 2, 4, 8
 
 EXPORTS = ("bf1_route_capacity", "bf1_plan_route", "bf1_attn_fwd", "bf1_dense_causal_fwd",
-           "bf1_last_error", "bf1_version")
+           "bf1_attn_fwd_noalloc", "bf1_last_error", "bf1_version")
 
 
 class RouteCfg(ctypes.Structure):
@@ -66,6 +66,9 @@ def load():
     L.bf1_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(_RouteC), vp, vp, vp]
     L.bf1_dense_causal_fwd.restype = ctypes.c_int
     L.bf1_dense_causal_fwd.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, vp, vp, vp, vp]
+    L.bf1_attn_fwd_noalloc.restype = ctypes.c_int
+    L.bf1_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(RouteCfg),
+                                       vp, vp, vp, vp]
     L.bf1_last_error.restype = ctypes.c_char_p
     L.bf1_last_error.argtypes = []
     L.bf1_version.restype = ctypes.c_int
@@ -188,6 +191,24 @@ def dense_causal_fwd(q, k, v, cu_seqlens, max_seqlen: int, scale: Optional[float
                                        cu_seqlens.numel() - 1, T, max_seqlen, hq, hkv, d,
                                        float(scale) if scale else 0.0, out.data_ptr(), lse.data_ptr(),
                                        work.data_ptr() if work is not None else None,
+                                       _stream_ptr(stream)))
+    return out, lse
+
+
+def attn_fwd_noalloc(q, k, v, cu_seqlens, max_seqlen: int, out, lse, cfg: Optional[RouteCfg] = None,
+                     scale: Optional[float] = None, status=None, stream=None):
+    """bf1_attn_fwd_noalloc: plan + attention using the library's built-in scratch array.
+
+    For callers that must not allocate device memory, so `out` and `lse` are required here and
+    the call itself allocates nothing (neither through torch nor through CUDA).  Up to 4096
+    query blocks per batch; calls sharing a GPU must not overlap in time."""
+    T, hq, hkv, d = _check_qkv(q, k, v)
+    cfg = cfg or RouteCfg()
+    total = getattr(cu_seqlens, "_bf1_total", T)
+    _check(load().bf1_attn_fwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), cu_seqlens.data_ptr(),
+                                       cu_seqlens.numel() - 1, total, max_seqlen, hq, hkv, d,
+                                       float(scale) if scale else 0.0, ctypes.byref(cfg), out.data_ptr(),
+                                       lse.data_ptr(), status.data_ptr() if status is not None else None,
                                        _stream_ptr(stream)))
     return out, lse
 
