@@ -60,10 +60,12 @@ struct Cfg {
     static constexpr int kChunks = D / 64;                 // 128-byte column chunks per row
     static constexpr int kQBytes = kRows * D * 2;          // 32 KB at d = 128
     static constexpr int kTileBytes = kBlock * D * 2;      // one K or V block: 16 KB at d = 128
-    static constexpr int kRing = (D == 128) ? 5 : 8;       // ring slots
+    static constexpr int kRing = (D == 128) ? 4 : 8;       // ring slots
+    static constexpr int kStageBytes = kRows * 128;        // O staging: 128 rows x one 64-column chunk
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = kQBytes;
-    static constexpr int kBarOff = kRingOff + kRing * kTileBytes;
+    static constexpr int kStageOff = kRingOff + kRing * kTileBytes;
+    static constexpr int kBarOff = kStageOff + kStageBytes;
     static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1 + 2;
     static constexpr int kMiscOff = kBarOff + 8 * kNumBars;
     static constexpr int kInfoOff = kMiscOff + 16;             // two int4 unit descriptors
@@ -143,6 +145,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k,
                                                                const __grid_constant__ CUtensorMap tm_v,
+                                                               const __grid_constant__ CUtensorMap tm_o,
                                                                const AttnArgs args) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -171,6 +174,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const uint32_t base = smem_u32(smem);
     const uint32_t sQ = base + C::kQOff;
     const uint32_t sRing = base + C::kRingOff;
+    const uint32_t sStage = base + C::kStageOff;
     const uint32_t bar_q_full = base + C::kBarOff;
     const uint32_t bar_q_free = bar_q_full + 8;
     const uint32_t bar_full = bar_q_free + 8;                 // [kRing]
@@ -217,6 +221,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
     }
     __syncwarp();
     if (warp == 1) {
@@ -233,80 +238,124 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
 
     if (warp == 0) {
         // ================================ TMA producer ====================================
-        if (lane == 0) {
+        // The whole warp walks the loop; one elected lane issues the copies.  The 32 lanes fetch
+        // (and range-check) 32 list entries with one coalesced load and hand them round by shuffle.
+        {
             int slot = 0, pass = 0;
             Tracer tr;
-            tr.init(0);
+            if (lane == 0) tr.init(0);
             int n_tiles = 0;
             (void)n_tiles;
             auto next_unit = [&](int n) -> int {
-                return args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
+                int u = 0;
+                if (lane == 0) u = args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
+                return __shfl_sync(0xffffffffu, u, 0);
+            };
+            // entries [base, base + 32) of the unit's list, one per lane, made safe to use
+            auto fetch_entries = [&](const Unit& x, int base_i) -> int {
+                const int i = base_i + lane;
+                if (i >= x.cnt) return 0;
+                int p = args.dense ? i : x.list[i];
+                if (p < 0 || p > x.j || (i == x.cnt - 1) != (p == x.j)) {   // stay inside the sequence
+                    if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
+                    p = (i == x.cnt - 1) ? x.j : 0;
+                }
+                return p;
+            };
+            // Pull the unit's Q and (first 32) K/V blocks into L2 ahead of the real loads: TMA
+            // prefetches need no shared memory, and each lane issues the ones for its own entry.
+            auto prefetch_l2 = [&](const Unit& x, int my_p) {
+                if (lane < 2) {
+#pragma unroll
+                    for (int c = 0; c < C::kChunks; ++c) tma_prefetch_l2_3d(&tm_q, c * 64, x.kvh * 2 + lane, x.tok0);
+                }
+                if (lane < x.cnt) {
+                    const int row = x.seq0 + my_p * kBlock;
+#pragma unroll
+                    for (int c = 0; c < C::kChunks; ++c) {
+                        tma_prefetch_l2_3d(&tm_k, c * 64, x.kvh, row);
+                        tma_prefetch_l2_3d(&tm_v, c * 64, x.kvh, row);
+                    }
+                }
             };
             Unit un = {};
             bool have = false;
+            int my_p = 0;
             {
                 const int u = next_unit(0);
                 have = u < total_units;
-                if (have) decode_unit(args, nqb, u, un);
-            }
-            for (int n = 0;; ++n) {
-                if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
-                if (*abort_flag) have = false;
-                TR(tr, 1, n);
-                // publish the unit (or the end marker cnt = 0) to the other roles
-                s_info[n & 1].x = have ? un.cnt : 0;
-                s_info[n & 1].y = un.rows_valid;
-                s_info[n & 1].z = un.tok0;
-                s_info[n & 1].w = un.kvh;
-                mbar_arrive(bar_info + 8 * (n & 1));
-                if (!have) {
-                    mbar_arrive(bar_q_full);
-                    break;
+                if (have) {
+                    decode_unit(args, nqb, u, un);
+                    my_p = fetch_entries(un, 0);
                 }
-                mbar_expect_tx(bar_q_full, C::kQBytes);
-#pragma unroll
-                for (int c = 0; c < C::kChunks; ++c)
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_3d(sQ + c * (kRows * 128) + h * (kBlock * 128), &tm_q, c * 64, un.kvh * 2 + h,
-                                    un.tok0, bar_q_full);
-                auto entry = [&](int i) -> int {
-                    int p = args.dense ? i : un.list[i];
-                    if (p < 0 || p > un.j || (i == un.cnt - 1) != (p == un.j)) {   // stay inside the sequence
-                        if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
-                        p = (i == un.cnt - 1) ? un.j : 0;
-                    }
-                    return p;
-                };
-                auto load_tile = [&](int p, bool is_v) {
-                    if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
-                    const uint32_t bar = bar_full + 8 * slot;
-                    TR(tr, 2, n_tiles++);
+            }
+            auto load_tile = [&](int p, bool is_v) {
+                if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
+                const uint32_t bar = bar_full + 8 * slot;
+                TR(tr, 2, n_tiles++);
+                if (elect_one()) {
                     mbar_expect_tx(bar, C::kTileBytes);
                     const uint32_t dst = sRing + slot * C::kTileBytes;
                     const int row = un.seq0 + p * kBlock;
 #pragma unroll
                     for (int c = 0; c < C::kChunks; ++c)
                         tma_load_3d(dst + c * (kBlock * 128), is_v ? &tm_v : &tm_k, c * 64, un.kvh, row, bar);
-                    if (++slot == C::kRing) { slot = 0; ++pass; }
-                };
-                // K0, K1, V0, K2, V1, ...: the order in which the MMA warp consumes them; list
-                // entries are fetched one tile ahead so that their latency hides behind the ring waits
-                int p_prev = entry(0);
-                int p_cur = un.cnt > 1 ? entry(1) : 0;
-                load_tile(p_prev, false);
+                }
+                __syncwarp();
+                if (++slot == C::kRing) { slot = 0; ++pass; }
+            };
+            for (int n = 0;; ++n) {
+                // K0 of this unit only needs a ring slot, not the Q buffer: get it going first
+                int base_i = 0;
+                int p_prev = 0;
+                if (have) {
+                    p_prev = __shfl_sync(0xffffffffu, my_p, 0);
+                    load_tile(p_prev, false);
+                }
+                if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
+                if (*abort_flag) have = false;
+                TR(tr, 1, n);
+                if (elect_one()) {
+                    // publish the unit (or the end marker cnt = 0) to the other roles
+                    s_info[n & 1].x = have ? un.cnt : 0;
+                    s_info[n & 1].y = un.rows_valid;
+                    s_info[n & 1].z = un.tok0;
+                    s_info[n & 1].w = un.kvh;
+                    mbar_arrive(bar_info + 8 * (n & 1));
+                    if (!have) {
+                        mbar_arrive(bar_q_full);
+                    } else {
+                        mbar_expect_tx(bar_q_full, C::kQBytes);
+#pragma unroll
+                        for (int c = 0; c < C::kChunks; ++c)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_3d(sQ + c * (kRows * 128) + h * (kBlock * 128), &tm_q, c * 64,
+                                            un.kvh * 2 + h, un.tok0, bar_q_full);
+                    }
+                }
+                __syncwarp();
+                if (!have) break;
+                // K1, V0, K2, V1, ...: the order in which the MMA warp consumes them
                 for (int i = 1; i < un.cnt; ++i) {
-                    const int p_next = (i + 1 < un.cnt) ? entry(i + 1) : 0;
+                    if (i - base_i == 32) {   // lists longer than a warp: next batch of entries
+                        base_i += 32;
+                        my_p = fetch_entries(un, base_i);
+                    }
+                    const int p_cur = __shfl_sync(0xffffffffu, my_p, i - base_i);
                     load_tile(p_cur, false);
                     load_tile(p_prev, true);
                     p_prev = p_cur;
-                    p_cur = p_next;
                 }
                 load_tile(p_prev, true);
-                // decode the next unit now: the loads overlap the wait for the Q buffer
+                // fetch and decode the next unit now; its loads overlap the wait for the Q buffer
                 const int u = next_unit(n + 1);
                 have = u < total_units;
-                if (have) decode_unit(args, nqb, u, un);
+                if (have) {
+                    decode_unit(args, nqb, u, un);
+                    my_p = fetch_entries(un, 0);
+                    prefetch_l2(un, my_p);
+                }
                 TR(tr, 3, n);
             }
         }
@@ -493,27 +542,50 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             const float inv_l = 1.f / l_run;
             const int tok = un.tok0 + tl;
             const bool store = tl < un.rows_valid;
+            const bool full_tile = un.rows_valid == kBlock;   // CTA-uniform
             __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (un.kvh * 2 + hl)) * D;
+            const bool issuer = (warp == 2 && lane == 0);
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t oreg[32];
-                tmem_ld32(t_lane + C::kColO + c * 32, oreg);
+            for (int dc = 0; dc < C::kChunks; ++dc) {
+                uint32_t oreg[64];
+                {
+                    uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&oreg[0]);
+                    uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&oreg[32]);
+                    tmem_ld32(t_lane + C::kColO + dc * 64, lo);
+                    tmem_ld32(t_lane + C::kColO + dc * 64 + 32, hi);
+                }
                 tmem_wait_ld();
-                if (c == D / 32 - 1) {   // O has been read out: the next unit may overwrite it
+                if (dc == C::kChunks - 1) {   // O has been read out: the next unit may overwrite it
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_o_free);
                 }
-                if (store) {
+                uint32_t w[32];
 #pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(oreg[e + 0]) * inv_l, __uint_as_float(oreg[e + 1]) * inv_l);
-                        w.y = pack_bf16x2(__uint_as_float(oreg[e + 2]) * inv_l, __uint_as_float(oreg[e + 3]) * inv_l);
-                        w.z = pack_bf16x2(__uint_as_float(oreg[e + 4]) * inv_l, __uint_as_float(oreg[e + 5]) * inv_l);
-                        w.w = pack_bf16x2(__uint_as_float(oreg[e + 6]) * inv_l, __uint_as_float(oreg[e + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + e) = w;
+                for (int e = 0; e < 32; ++e)
+                    w[e] = pack_bf16x2(__uint_as_float(oreg[2 * e]) * inv_l, __uint_as_float(oreg[2 * e + 1]) * inv_l);
+                if (full_tile) {
+                    // Full block: rows go to a swizzled staging tile (one 64-column chunk of both heads)
+                    // and leave through two TMA stores, so nobody waits for scattered global writes.
+                    if (issuer) bulk_wait_read0();       // the previous store has finished reading the tile
+                    named_barrier(1, 128);
+                    const uint32_t srow = sStage + hl * (kBlock * 128) + tl * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        st_shared_v4(srow + ((c ^ (tl & 7)) << 4), w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                    fence_proxy_async();
+                    named_barrier(1, 128);
+                    if (issuer) {
+                        tma_store_3d(&tm_o, dc * 64, un.kvh * 2 + 0, un.tok0, sStage);
+                        tma_store_3d(&tm_o, dc * 64, un.kvh * 2 + 1, un.tok0, sStage + kBlock * 128);
+                        bulk_commit_group();
                     }
+                } else if (store) {
+                    // partial last block of a sequence: the rows after it belong to someone else
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4*>(orow + dc * 64 + c * 8) =
+                            make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
                 }
             }
             if (store) {
@@ -523,6 +595,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         }
     }
 
+    if (warp == 2 && lane == 0) bulk_wait0();   // this thread's output stores have landed
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
@@ -622,7 +695,8 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     DeviceInfo info;
     if (int rc = device_info(&info)) return rc;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
+    if (int rc = make_map(&to, o, total_tokens, hq, d)) return rc;
     if (int rc = make_map(&tq, q, total_tokens, hq, d)) return rc;
     if (int rc = make_map(&tk, k, total_tokens, hkv, d)) return rc;
     if (int rc = make_map(&tv, v, total_tokens, hkv, d)) return rc;
@@ -652,9 +726,9 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     const int64_t units = slots * hkv;
     const int grid = (int)(units < 2LL * info.sm_count ? units : 2LL * info.sm_count);
     if (d == 128)
-        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
+        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);
     else
-        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
+        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
 }
