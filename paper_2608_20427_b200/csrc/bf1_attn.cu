@@ -13,13 +13,19 @@
 // then O / l is written as bf16 and LSE = max + ln(sum) as fp32.
 // With `dense = 1` the list is replaced by 0..j: plain causal attention through the same code.
 //
-// The kernel is persistent (two CTAs per SM, each walking a strided share of the units in
-// longest-list-first order) and warp specialised:
-//   warp 0     TMA producer: Q once per unit, then K and V tiles through a ring of 16 KB slots
-//              in the order the MMAs consume them (K0, K1, V0, K2, V1, ...),
-//   warp 1     MMA issuer: S(g+1) is issued before PV(g), so the tensor pipe works on the next
-//              tile's scores and the previous tile's PV while the softmax warps are busy,
-//   warps 2-5  softmax + epilogue, one thread per tile row.
+// The kernel is persistent (two CTAs per SM; units are handed out KV-head-major, longest list
+// first, through an atomic counter) and warp specialised, 12 warps in three warpgroups whose
+// register budgets are re-balanced with setmaxnreg:
+//   warp 0      TMA producer: Q once per unit, then K and V tiles through a ring of 16 KB slots
+//               in the order the MMAs consume them (K0, K1, V0, K2, V1, ...),
+//   warp 1      MMA issuer: S(g+1) is issued before PV(g), so the tensor pipe works on the next
+//               tile's scores and the previous tile's PV while the softmax warps are busy,
+//   warp 2      scheduler: fetches the next unit, decodes it, reads (and range-checks) its list,
+//               prefetches its Q/K/V blocks into L2 and queues it for the producer -- all of it
+//               global-memory latency that must not sit in front of the copies,
+//   warps 4-7   softmax, one thread per tile row,
+//   warps 8-11  epilogue: take the finished O out of tensor memory, normalise, store O and LSE,
+//               while the softmax warps are already on the next unit.
 // All hand-offs are mbarriers; every wait is bounded (see mbar_wait).
 #include <cuda.h>
 
@@ -29,7 +35,19 @@ namespace bf1 {
 
 constexpr int kBlock = 64;            // b: tokens per block
 constexpr int kRows = 128;            // MMA M: 2 query heads x 64 tokens
-constexpr int kThreads = 192;         // 6 warps
+constexpr int kThreads = 384;         // 12 warps
+constexpr int kQueue = 3;             // decoded units queued between scheduler and producer
+#ifndef BF1_REGS_CTL
+#define BF1_REGS_CTL 40
+#define BF1_REGS_SOFTMAX 144
+#define BF1_REGS_EPILOGUE 56
+#endif
+constexpr int kRegsCtl = BF1_REGS_CTL, kRegsSoftmax = BF1_REGS_SOFTMAX, kRegsEpilogue = BF1_REGS_EPILOGUE;
+static_assert(kRegsCtl + kRegsSoftmax + kRegsEpilogue <= 240, "register budgets must fit the launch allocation");
+#ifndef BF1_PREFETCH_MODE
+#define BF1_PREFETCH_MODE 0
+#endif
+constexpr int kPrefetchMode = BF1_PREFETCH_MODE;   // L2 prefetch of queued units: 0 none, 1 Q only, 2 Q + K/V
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row
                                             // maximum grows by more than 2^8
 
@@ -55,21 +73,34 @@ struct AttnArgs {
     float* lse;
 };
 
+// One decoded unit as the scheduler queues it for the producer.
+struct QueueEntry {
+    int32_t cnt, rows_valid, tok0, kvh, seq0, j, slot, pad;
+    int32_t p[32];         // first 32 list entries, range-checked
+};
+
+// What the softmax warps leave for the epilogue warps when a unit's last tile is done.
+struct Handoff {
+    float m[kRows];        // reference maximum per row (raw score units)
+    float l[kRows];        // sum of exp2((s - m) * scale_log2) per row
+    int32_t cnt, rows_valid, tok0, kvh, g_last, pad[3];
+};
+
 template <int D>
 struct Cfg {
     static constexpr int kChunks = D / 64;                 // 128-byte column chunks per row
     static constexpr int kQBytes = kRows * D * 2;          // 32 KB at d = 128
     static constexpr int kTileBytes = kBlock * D * 2;      // one K or V block: 16 KB at d = 128
     static constexpr int kRing = (D == 128) ? 4 : 8;       // ring slots
-    static constexpr int kStageBytes = kRows * 128;        // O staging: 128 rows x one 64-column chunk
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = kQBytes;
-    static constexpr int kStageOff = kRingOff + kRing * kTileBytes;
-    static constexpr int kBarOff = kStageOff + kStageBytes;
-    static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1 + 2;
+    static constexpr int kHandOff = kRingOff + kRing * kTileBytes;          // Handoff[2]
+    static constexpr int kQueueOff = kHandOff + 2 * (int)sizeof(Handoff);   // QueueEntry[kQueue]
+    static constexpr int kInfoOff = kQueueOff + kQueue * (int)sizeof(QueueEntry);   // int4[2]
+    static constexpr int kBarOff = kInfoOff + 32;
+    static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1 + 2 + 2 * kQueue + 2 + 2;
     static constexpr int kMiscOff = kBarOff + 8 * kNumBars;
-    static constexpr int kInfoOff = kMiscOff + 16;             // two int4 unit descriptors
-    static constexpr int kTotal = kInfoOff + 32;
+    static constexpr int kTotal = kMiscOff + 16;
     static constexpr int kTmemCols = 256;
     static constexpr int kColS = 0;                        // S buffers: 2 x 64 fp32 columns
     static constexpr int kColO = 128;                      // O: D fp32 columns
@@ -105,7 +136,7 @@ struct Tracer {
 #endif
 
 struct Unit {
-    int seq0, j, cnt, rows_valid, kvh, tok0;
+    int seq0, j, cnt, rows_valid, kvh, tok0, slot;
     const int32_t* list;
 };
 
@@ -121,6 +152,7 @@ __device__ __forceinline__ void decode_unit(const AttnArgs& a, int nqb, int u, U
         un.j = a.qb_block[slot];
         int c = a.kv_count[slot];
         un.cnt = min(max(c, 1), a.max_degree);
+        un.slot = slot;
         un.list = a.kv_idx + (size_t)slot * a.max_degree;
     } else {
         slot = nqb - 1 - idx;
@@ -133,6 +165,7 @@ __device__ __forceinline__ void decode_unit(const AttnArgs& a, int nqb, int u, U
             acc += nb;
         }
         un.cnt = un.j + 1;
+        un.slot = slot;
         un.list = nullptr;
     }
     un.seq0 = a.cu_seqlens[seq];
@@ -141,11 +174,19 @@ __device__ __forceinline__ void decode_unit(const AttnArgs& a, int nqb, int u, U
     un.tok0 = un.seq0 + un.j * kBlock;
 }
 
+template <int REGS>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS));
+}
+template <int REGS>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS));
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k,
                                                                const __grid_constant__ CUtensorMap tm_v,
-                                                               const __grid_constant__ CUtensorMap tm_o,
                                                                const AttnArgs args) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -174,7 +215,6 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const uint32_t base = smem_u32(smem);
     const uint32_t sQ = base + C::kQOff;
     const uint32_t sRing = base + C::kRingOff;
-    const uint32_t sStage = base + C::kStageOff;
     const uint32_t bar_q_full = base + C::kBarOff;
     const uint32_t bar_q_free = bar_q_full + 8;
     const uint32_t bar_full = bar_q_free + 8;                 // [kRing]
@@ -184,7 +224,13 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const uint32_t bar_pv_done = bar_p_full + 16;             // [2]
     const uint32_t bar_o_free = bar_pv_done + 16;
     const uint32_t bar_info = bar_o_free + 8;                 // [2]
+    const uint32_t bar_sq_full = bar_info + 16;               // [kQueue]
+    const uint32_t bar_sq_free = bar_sq_full + 8 * kQueue;    // [kQueue]
+    const uint32_t bar_ho_full = bar_sq_free + 8 * kQueue;    // [2]
+    const uint32_t bar_ho_free = bar_ho_full + 16;            // [2]
     volatile int4* s_info = reinterpret_cast<volatile int4*>(smem + C::kInfoOff);   // {cnt, rows_valid, tok0, kvh}
+    volatile QueueEntry* s_queue = reinterpret_cast<volatile QueueEntry*>(smem + C::kQueueOff);
+    volatile Handoff* s_hand = reinterpret_cast<volatile Handoff*>(smem + C::kHandOff);
     uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + C::kMiscOff);
     int* s_abort = reinterpret_cast<int*>(smem + C::kMiscOff + 4);
     int* s_nqb = reinterpret_cast<int*>(smem + C::kMiscOff + 8);
@@ -213,15 +259,19 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             mbar_init(bar_s_full + 8 * s, 1);
             mbar_init(bar_p_full + 8 * s, 4);    // one arrival per softmax warp
             mbar_init(bar_pv_done + 8 * s, 1);
+            mbar_init(bar_info + 8 * s, 1);
+            mbar_init(bar_ho_full + 8 * s, 4);   // softmax warps
+            mbar_init(bar_ho_free + 8 * s, 4);   // epilogue warps
         }
-        mbar_init(bar_o_free, 4);
-        mbar_init(bar_info, 1);
-        mbar_init(bar_info + 8, 1);
+        for (int s = 0; s < kQueue; ++s) {
+            mbar_init(bar_sq_full + 8 * s, 1);
+            mbar_init(bar_sq_free + 8 * s, 1);
+        }
+        mbar_init(bar_o_free, 4);                // epilogue warps
         fence_mbar_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
-        tma_prefetch_desc(&tm_o);
     }
     __syncwarp();
     if (warp == 1) {
@@ -236,111 +286,118 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const int nqb = *s_nqb;
     const int total_units = nqb * args.hkv;
 
-    if (warp == 0) {
-        // ================================ TMA producer ====================================
-        // The whole warp walks the loop; one elected lane issues the copies.  The 32 lanes fetch
-        // (and range-check) 32 list entries with one coalesced load and hand them round by shuffle.
-        {
+    if (warp < 4) {
+        setmaxnreg_dec<kRegsCtl>();
+        if (warp == 2) {
+            // ================================ scheduler =======================================
+            for (int n = 0;; ++n) {
+                int u = 0;
+                if (lane == 0) u = args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
+                u = __shfl_sync(0xffffffffu, u, 0);
+                const bool have = u < total_units && !*abort_flag;
+                Unit un = {};
+                int my_p = 0;
+                if (have) {
+                    decode_unit(args, nqb, u, un);
+                    if (lane < un.cnt) {   // entries 0..31, one per lane, made safe to use
+                        int p = args.dense ? lane : un.list[lane];
+                        if (p < 0 || p > un.j || (lane == un.cnt - 1) != (p == un.j)) {
+                            if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
+                            p = (lane == un.cnt - 1) ? un.j : 0;
+                        }
+                        my_p = p;
+                        if (kPrefetchMode >= 2) {
+                            // pull this block into L2 ahead of the real load (needs no shared memory)
+                            const int row = un.seq0 + p * kBlock;
+                            tma_prefetch_l2_4d(&tm_k, 0, row, un.kvh, 0);
+                            tma_prefetch_l2_4d(&tm_v, 0, row, un.kvh, 0);
+                        }
+                    }
+                    if (kPrefetchMode >= 1 && lane == 0) tma_prefetch_l2_4d(&tm_q, 0, un.tok0, un.kvh * 2, 0);
+                }
+                const int qs = n % kQueue;
+                if (n >= kQueue) mbar_wait(bar_sq_free + 8 * qs, ((n / kQueue) - 1) & 1, abort_flag, args.status);
+                volatile QueueEntry* e = s_queue + qs;
+                e->p[lane] = my_p;
+                if (lane == 0) {
+                    e->cnt = have ? un.cnt : 0;
+                    e->rows_valid = un.rows_valid;
+                    e->tok0 = un.tok0;
+                    e->kvh = un.kvh;
+                    e->seq0 = un.seq0;
+                    e->j = un.j;
+                    e->slot = un.slot;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_sq_full + 8 * qs);
+                if (!have) break;
+            }
+        } else if (warp == 0) {
+            // ================================ TMA producer ====================================
+            // The whole warp walks the loop; one elected lane issues the copies.
             int slot = 0, pass = 0;
             Tracer tr;
             if (lane == 0) tr.init(0);
             int n_tiles = 0;
             (void)n_tiles;
-            auto next_unit = [&](int n) -> int {
-                int u = 0;
-                if (lane == 0) u = args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
-                return __shfl_sync(0xffffffffu, u, 0);
-            };
-            // entries [base, base + 32) of the unit's list, one per lane, made safe to use
-            auto fetch_entries = [&](const Unit& x, int base_i) -> int {
-                const int i = base_i + lane;
-                if (i >= x.cnt) return 0;
-                int p = args.dense ? i : x.list[i];
-                if (p < 0 || p > x.j || (i == x.cnt - 1) != (p == x.j)) {   // stay inside the sequence
-                    if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
-                    p = (i == x.cnt - 1) ? x.j : 0;
-                }
-                return p;
-            };
-            // Pull the unit's Q and (first 32) K/V blocks into L2 ahead of the real loads: TMA
-            // prefetches need no shared memory, and each lane issues the ones for its own entry.
-            auto prefetch_l2 = [&](const Unit& x, int my_p) {
-                if (lane < 2) {
-#pragma unroll
-                    for (int c = 0; c < C::kChunks; ++c) tma_prefetch_l2_3d(&tm_q, c * 64, x.kvh * 2 + lane, x.tok0);
-                }
-                if (lane < x.cnt) {
-                    const int row = x.seq0 + my_p * kBlock;
-#pragma unroll
-                    for (int c = 0; c < C::kChunks; ++c) {
-                        tma_prefetch_l2_3d(&tm_k, c * 64, x.kvh, row);
-                        tma_prefetch_l2_3d(&tm_v, c * 64, x.kvh, row);
-                    }
-                }
-            };
-            Unit un = {};
-            bool have = false;
-            int my_p = 0;
-            {
-                const int u = next_unit(0);
-                have = u < total_units;
-                if (have) {
-                    decode_unit(args, nqb, u, un);
-                    my_p = fetch_entries(un, 0);
-                }
-            }
-            auto load_tile = [&](int p, bool is_v) {
-                if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
-                const uint32_t bar = bar_full + 8 * slot;
-                TR(tr, 2, n_tiles++);
-                if (elect_one()) {
-                    mbar_expect_tx(bar, C::kTileBytes);
-                    const uint32_t dst = sRing + slot * C::kTileBytes;
-                    const int row = un.seq0 + p * kBlock;
-#pragma unroll
-                    for (int c = 0; c < C::kChunks; ++c)
-                        tma_load_3d(dst + c * (kBlock * 128), is_v ? &tm_v : &tm_k, c * 64, un.kvh, row, bar);
-                }
-                __syncwarp();
-                if (++slot == C::kRing) { slot = 0; ++pass; }
-            };
             for (int n = 0;; ++n) {
-                // K0 of this unit only needs a ring slot, not the Q buffer: get it going first
-                int base_i = 0;
-                int p_prev = 0;
-                if (have) {
-                    p_prev = __shfl_sync(0xffffffffu, my_p, 0);
-                    load_tile(p_prev, false);
-                }
+                const int qs = n % kQueue;
+                mbar_wait(bar_sq_full + 8 * qs, (n / kQueue) & 1, abort_flag, args.status);
+                volatile QueueEntry* e = s_queue + qs;
+                int cnt = e->cnt;
+                const int rows_valid = e->rows_valid, tok0 = e->tok0, kvh = e->kvh, seq0 = e->seq0, j = e->j;
+                const int rslot = e->slot;
+                int my_p = e->p[lane];
+                if (*abort_flag) cnt = 0;
+                auto load_tile = [&](int p, bool is_v) {
+                    if (pass > 0) mbar_wait(bar_free + 8 * slot, (pass - 1) & 1, abort_flag, args.status);
+                    const uint32_t bar = bar_full + 8 * slot;
+                    TR(tr, 2, n_tiles++);
+                    if (elect_one()) {
+                        mbar_expect_tx(bar, C::kTileBytes);
+                        // one copy per tile: box = 64 elements x 64 tokens x 1 head x all column chunks
+                        tma_load_4d(sRing + slot * C::kTileBytes, is_v ? &tm_v : &tm_k, 0, seq0 + p * kBlock, kvh, 0, bar);
+                    }
+                    __syncwarp();
+                    if (++slot == C::kRing) { slot = 0; ++pass; }
+                };
+                // K0 only needs a ring slot, not the Q buffer: get it going first
+                int p_prev = __shfl_sync(0xffffffffu, my_p, 0);
+                if (cnt > 0) load_tile(p_prev, false);
                 if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
-                if (*abort_flag) have = false;
                 TR(tr, 1, n);
                 if (elect_one()) {
-                    // publish the unit (or the end marker cnt = 0) to the other roles
-                    s_info[n & 1].x = have ? un.cnt : 0;
-                    s_info[n & 1].y = un.rows_valid;
-                    s_info[n & 1].z = un.tok0;
-                    s_info[n & 1].w = un.kvh;
+                    // publish the unit (or the end marker cnt = 0) to the MMA and softmax warps
+                    s_info[n & 1].x = cnt;
+                    s_info[n & 1].y = rows_valid;
+                    s_info[n & 1].z = tok0;
+                    s_info[n & 1].w = kvh;
                     mbar_arrive(bar_info + 8 * (n & 1));
-                    if (!have) {
+                    if (cnt == 0) {
                         mbar_arrive(bar_q_full);
                     } else {
                         mbar_expect_tx(bar_q_full, C::kQBytes);
-#pragma unroll
-                        for (int c = 0; c < C::kChunks; ++c)
-#pragma unroll
-                            for (int h = 0; h < 2; ++h)
-                                tma_load_3d(sQ + c * (kRows * 128) + h * (kBlock * 128), &tm_q, c * 64,
-                                            un.kvh * 2 + h, un.tok0, bar_q_full);
+                        // one copy: box = 64 elements x 64 tokens x 2 heads x all column chunks
+                        tma_load_4d(sQ, &tm_q, 0, tok0, kvh * 2, 0, bar_q_full);
                     }
                 }
                 __syncwarp();
-                if (!have) break;
+                if (cnt == 0) break;
                 // K1, V0, K2, V1, ...: the order in which the MMA warp consumes them
-                for (int i = 1; i < un.cnt; ++i) {
-                    if (i - base_i == 32) {   // lists longer than a warp: next batch of entries
+                int base_i = 0;
+                for (int i = 1; i < cnt; ++i) {
+                    if (i - base_i == 32) {   // lists longer than a warp: fetch the next 32 entries
                         base_i += 32;
-                        my_p = fetch_entries(un, base_i);
+                        const int ii = base_i + lane;
+                        int p = 0;
+                        if (ii < cnt) {
+                            p = args.dense ? ii : args.kv_idx[(size_t)rslot * args.max_degree + ii];
+                            if (p < 0 || p > j || (ii == cnt - 1) != (p == j)) {
+                                if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
+                                p = (ii == cnt - 1) ? j : 0;
+                            }
+                        }
+                        my_p = p;
                     }
                     const int p_cur = __shfl_sync(0xffffffffu, my_p, i - base_i);
                     load_tile(p_cur, false);
@@ -348,23 +405,14 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     p_prev = p_cur;
                 }
                 load_tile(p_prev, true);
-                // fetch and decode the next unit now; its loads overlap the wait for the Q buffer
-                const int u = next_unit(n + 1);
-                have = u < total_units;
-                if (have) {
-                    decode_unit(args, nqb, u, un);
-                    my_p = fetch_entries(un, 0);
-                    prefetch_l2(un, my_p);
-                }
+                if (elect_one()) mbar_arrive(bar_sq_free + 8 * qs);
+                __syncwarp();
                 TR(tr, 3, n);
             }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ================================ MMA issuer ======================================
-        // The whole warp walks the loop (so that addresses and descriptors stay warp-uniform and
-        // cheap); one elected lane issues the MMAs and commits.
-        {
+        } else if (warp == 1) {
+            // ================================ MMA issuer ======================================
+            // The whole warp walks the loop (so that addresses and descriptors stay warp-uniform and
+            // cheap); one elected lane issues the MMAs and commits.
             constexpr uint32_t kIdescS = idesc_bf16_f32(kBlock, false);   // 128 x 64 x 16, K-major B
             constexpr uint32_t kIdescO = idesc_bf16_f32(D, true);         // 128 x D x 16, MN-major B
             int slot = 0, pass = 0, n = 0;
@@ -439,31 +487,26 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             }
         }
         __syncwarp();
-    } else {
-        // ================================ softmax + epilogue ===============================
+    } else if (warp < 8) {
+        // ================================ softmax ==========================================
+        setmaxnreg_inc<kRegsSoftmax>();
         const int quarter = warp & 3;                     // TMEM lanes this warp may touch
         const int row = quarter * 32 + lane;              // tile row of this thread
-        const int hl = row >> 6;                          // which head of the pair
         const int tl = row & 63;                          // token inside the query block
         const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const float c2 = args.scale_log2;
         uint32_t g = 0;
-        int n = 0;
         Tracer tr;
-        if (warp == 2 && lane == 0) tr.init(2);
-        for (;; ++n) {
+        if (warp == 4 && lane == 0) tr.init(2);
+        for (int n = 0;; ++n) {
             TR(tr, 23, n);
             mbar_wait(bar_info + 8 * (n & 1), (n >> 1) & 1, abort_flag, args.status);
             TR(tr, 24, n);
-            Unit un;
-            un.cnt = s_info[n & 1].x;
-            un.rows_valid = s_info[n & 1].y;
-            un.tok0 = s_info[n & 1].z;
-            un.kvh = s_info[n & 1].w;
-            if (un.cnt == 0 || *abort_flag) break;
+            const int cnt = *abort_flag ? 0 : s_info[n & 1].x;
+            const int rows_valid = s_info[n & 1].y, tok0 = s_info[n & 1].z, kvh = s_info[n & 1].w;
             float m_used = 0.f;    // reference maximum (raw score units) the exponentials are taken against
             float l_run = 0.f;     // running sum of exp2((s - m_used) * c2)
-            for (int i = 0; i < un.cnt; ++i, ++g) {
+            for (int i = 0; i < cnt; ++i, ++g) {
                 const uint32_t t_s = t_lane + C::kColS + (g & 1) * 64;
                 mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);
                 TR(tr, 20, g);
@@ -476,7 +519,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     tmem_ld32(t_s + 32, hi);
                 }
                 tmem_wait_ld();
-                if (i == un.cnt - 1) {   // self block: causal triangle (warp-uniform branch)
+                if (i == cnt - 1) {   // self block: causal triangle (warp-uniform branch)
 #pragma unroll
                     for (int c = 0; c < 64; ++c)
                         if (c > tl) sreg[c] = 0xff800000u;   // -inf
@@ -526,8 +569,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 }
                 float r0, r1;
                 unpack2(add2(sum_a, sum_b), r0, r1);
-                const float rowsum = r0 + r1;
-                l_run += rowsum;
+                l_run += r0 + r1;
                 tmem_st32(t_s, preg);   // P overwrites the first 32 columns of this S buffer
                 tmem_wait_st();
                 tc_fence_before();
@@ -535,67 +577,80 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(bar_p_full + 8 * (g & 1));
                 TR(tr, 21, g);
             }
-            // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------
-            mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
+            // ---- hand the unit over to the epilogue warps -------------------------------------
+            if (n >= 2) mbar_wait(bar_ho_free + 8 * (n & 1), ((n >> 1) - 1) & 1, abort_flag, args.status);
+            volatile Handoff* h = s_hand + (n & 1);
+            h->m[row] = m_used;
+            h->l[row] = l_run;
+            if (row == 0) {
+                h->cnt = cnt;
+                h->rows_valid = rows_valid;
+                h->tok0 = tok0;
+                h->kvh = kvh;
+                h->g_last = (int)(g - 1);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ho_full + 8 * (n & 1));
             TR(tr, 22, n);
+            if (cnt == 0) break;
+        }
+    } else {
+        // ================================ epilogue =========================================
+        setmaxnreg_dec<kRegsEpilogue>();
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int hl = row >> 6;                          // which head of the pair
+        const int tl = row & 63;
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        const float c2 = args.scale_log2;
+        for (int n = 0;; ++n) {
+            mbar_wait(bar_ho_full + 8 * (n & 1), (n >> 1) & 1, abort_flag, args.status);
+            volatile Handoff* h = s_hand + (n & 1);
+            const float m_used = h->m[row], l_run = h->l[row];
+            const int cnt = *abort_flag ? 0 : h->cnt;
+            const int rows_valid = h->rows_valid, tok0 = h->tok0, kvh = h->kvh;
+            const uint32_t gl = (uint32_t)h->g_last;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ho_free + 8 * (n & 1));
+            if (cnt == 0) break;
+            mbar_wait(bar_pv_done + 8 * (gl & 1), (gl >> 1) & 1, abort_flag, args.status);
             tc_fence_after();
             const float inv_l = 1.f / l_run;
-            const int tok = un.tok0 + tl;
-            const bool store = tl < un.rows_valid;
-            const bool full_tile = un.rows_valid == kBlock;   // CTA-uniform
-            __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (un.kvh * 2 + hl)) * D;
-            const bool issuer = (warp == 2 && lane == 0);
+            const int tok = tok0 + tl;
+            const bool store = tl < rows_valid;
+            __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * 2 + hl)) * D;
+            // 16 columns at a time keeps this warpgroup inside its small register budget
 #pragma unroll
-            for (int dc = 0; dc < C::kChunks; ++dc) {
-                uint32_t oreg[64];
-                {
-                    uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&oreg[0]);
-                    uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&oreg[32]);
-                    tmem_ld32(t_lane + C::kColO + dc * 64, lo);
-                    tmem_ld32(t_lane + C::kColO + dc * 64 + 32, hi);
-                }
+            for (int c = 0; c < D / 16; ++c) {
+                uint32_t oreg[16];
+                tmem_ld16(t_lane + C::kColO + c * 16, oreg);
                 tmem_wait_ld();
-                if (dc == C::kChunks - 1) {   // O has been read out: the next unit may overwrite it
+                if (c == D / 16 - 1) {   // O has been read out: the next unit may overwrite it
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_o_free);
                 }
-                uint32_t w[32];
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    w[e] = pack_bf16x2(__uint_as_float(oreg[2 * e]) * inv_l, __uint_as_float(oreg[2 * e + 1]) * inv_l);
-                if (full_tile) {
-                    // Full block: rows go to a swizzled staging tile (one 64-column chunk of both heads)
-                    // and leave through two TMA stores, so nobody waits for scattered global writes.
-                    if (issuer) bulk_wait_read0();       // the previous store has finished reading the tile
-                    named_barrier(1, 128);
-                    const uint32_t srow = sStage + hl * (kBlock * 128) + tl * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        st_shared_v4(srow + ((c ^ (tl & 7)) << 4), w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-                    fence_proxy_async();
-                    named_barrier(1, 128);
-                    if (issuer) {
-                        tma_store_3d(&tm_o, dc * 64, un.kvh * 2 + 0, un.tok0, sStage);
-                        tma_store_3d(&tm_o, dc * 64, un.kvh * 2 + 1, un.tok0, sStage + kBlock * 128);
-                        bulk_commit_group();
-                    }
-                } else if (store) {
-                    // partial last block of a sequence: the rows after it belong to someone else
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<uint4*>(orow + dc * 64 + c * 8) =
-                            make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                if (store) {
+                    uint4 w0, w1;
+                    w0.x = pack_bf16x2(__uint_as_float(oreg[0]) * inv_l, __uint_as_float(oreg[1]) * inv_l);
+                    w0.y = pack_bf16x2(__uint_as_float(oreg[2]) * inv_l, __uint_as_float(oreg[3]) * inv_l);
+                    w0.z = pack_bf16x2(__uint_as_float(oreg[4]) * inv_l, __uint_as_float(oreg[5]) * inv_l);
+                    w0.w = pack_bf16x2(__uint_as_float(oreg[6]) * inv_l, __uint_as_float(oreg[7]) * inv_l);
+                    w1.x = pack_bf16x2(__uint_as_float(oreg[8]) * inv_l, __uint_as_float(oreg[9]) * inv_l);
+                    w1.y = pack_bf16x2(__uint_as_float(oreg[10]) * inv_l, __uint_as_float(oreg[11]) * inv_l);
+                    w1.z = pack_bf16x2(__uint_as_float(oreg[12]) * inv_l, __uint_as_float(oreg[13]) * inv_l);
+                    w1.w = pack_bf16x2(__uint_as_float(oreg[14]) * inv_l, __uint_as_float(oreg[15]) * inv_l);
+                    *reinterpret_cast<uint4*>(orow + c * 16) = w0;
+                    *reinterpret_cast<uint4*>(orow + c * 16 + 8) = w1;
                 }
             }
             if (store) {
                 const float lse2 = m_used * c2 + lg2_approx(l_run);   // log2 domain
-                args.lse[(size_t)(un.kvh * 2 + hl) * args.total_tokens + tok] = lse2 * 0.6931471805599453f;
+                args.lse[(size_t)(kvh * 2 + hl) * args.total_tokens + tok] = lse2 * 0.6931471805599453f;
             }
         }
     }
 
-    if (warp == 2 && lane == 0) bulk_wait0();   // this thread's output stores have landed
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
@@ -622,15 +677,18 @@ static int get_encode_fn(EncodeTiledFn* fn) {
     return BF1_OK;
 }
 
-// [T, H, d] bf16 tensor, box = 64 tokens x 1 head x 64 elements (128 bytes), 128-byte swizzle.
-static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d) {
+// [T, H, d] bf16 tensor seen as 4-D {64 elements, T tokens, H heads, d/64 column chunks}; box = 64
+// elements (128 bytes) x 64 tokens x `heads_per_box` heads x all chunks, 128-byte swizzle.  In shared
+// memory that is [chunk][head][token][128 B]: one K-major (or, for V, MN-major) 64-row tile per
+// chunk and head, which is what the MMA descriptors walk.
+static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box) {
     EncodeTiledFn enc;
     if (int rc = get_encode_fn(&enc)) return rc;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)T};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)H * d * 2};
-    cuuint32_t box[3] = {64, 1, (cuuint32_t)kBlock};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+    cuuint64_t dims[4] = {64, (cuuint64_t)T, (cuuint64_t)H, (cuuint64_t)(d / 64)};
+    cuuint64_t strides[3] = {(cuuint64_t)H * d * 2, (cuuint64_t)d * 2, 128};
+    cuuint32_t box[4] = {64, (cuuint32_t)kBlock, (cuuint32_t)heads_per_box, (cuuint32_t)(d / 64)};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(BF1_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -695,11 +753,10 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     DeviceInfo info;
     if (int rc = device_info(&info)) return rc;
 
-    CUtensorMap tq, tk, tv, to;
-    if (int rc = make_map(&to, o, total_tokens, hq, d)) return rc;
-    if (int rc = make_map(&tq, q, total_tokens, hq, d)) return rc;
-    if (int rc = make_map(&tk, k, total_tokens, hkv, d)) return rc;
-    if (int rc = make_map(&tv, v, total_tokens, hkv, d)) return rc;
+    CUtensorMap tq, tk, tv;
+    if (int rc = make_map(&tq, q, total_tokens, hq, d, 2)) return rc;
+    if (int rc = make_map(&tk, k, total_tokens, hkv, d, 1)) return rc;
+    if (int rc = make_map(&tv, v, total_tokens, hkv, d, 1)) return rc;
 
     AttnArgs a;
     a.cu_seqlens = cu_seqlens_dev;
@@ -726,9 +783,9 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     const int64_t units = slots * hkv;
     const int grid = (int)(units < 2LL * info.sm_count ? units : 2LL * info.sm_count);
     if (d == 128)
-        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);
+        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
     else
-        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);
+        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
 }
