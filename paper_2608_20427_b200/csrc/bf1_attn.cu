@@ -249,6 +249,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 nqb += (args.cu_seqlens[s + 1] - args.cu_seqlens[s] + kBlock - 1) / kBlock;
         }
         *s_nqb = nqb;
+        s_nqb[1] = 0;
         mbar_init(bar_q_full, 1);
         mbar_init(bar_q_free, 1);
         for (int s = 0; s < C::kRing; ++s) {
@@ -338,6 +339,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             int slot = 0, pass = 0;
             Tracer tr;
             if (lane == 0) tr.init(0);
+#ifdef BF1_TRACE
+            tr.cap = tr.cap / 2;   // the second half is the landing probe's
+#endif
             int n_tiles = 0;
             (void)n_tiles;
             for (int n = 0;; ++n) {
@@ -409,6 +413,24 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 __syncwarp();
                 TR(tr, 3, n);
             }
+#ifdef BF1_TRACE
+        } else if (warp == 3) {
+            // trace builds only: watch the ring's "full" barriers and record when each copy lands
+            if (lane == 0) {
+                Tracer tr;
+                tr.init(0);
+                tr.p = tr.p ? tr.p + 2 * (tr.cap / 2) : nullptr;   // second half of the producer's trace area
+                tr.cap = tr.cap / 2;
+                int slot = 0, pass = 0;
+                for (int e = 0;; ++e) {
+                    bool ok = false;
+                    while (!(ok = mbar_try_wait(bar_full + 8 * slot, pass & 1)) && !*(volatile int*)(s_nqb + 1)) {}
+                    if (!ok) break;
+                    TR(tr, 30, e);
+                    if (++slot == C::kRing) { slot = 0; ++pass; }
+                }
+            }
+#endif
         } else if (warp == 1) {
             // ================================ MMA issuer ======================================
             // The whole warp walks the loop (so that addresses and descriptors stay warp-uniform and
@@ -485,6 +507,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     if (++slot == C::kRing) { slot = 0; ++pass; }
                 }
             }
+#ifdef BF1_TRACE
+            if (lane == 0) *(volatile int*)(s_nqb + 1) = 1;   // tells the trace probe to stop
+#endif
         }
         __syncwarp();
     } else if (warp < 8) {
