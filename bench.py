@@ -159,6 +159,26 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ---- multi-rank bookkeeping (weak scaling: every rank runs its own copy, no data-path collective) --
+def rank_layer_seed_offset(rank: int, layer: int) -> int:
+    """Each rank draws its own inputs: rank r uses layers r*LAYERS .. r*LAYERS + LAYERS - 1."""
+    return layer + rank * LAYERS
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The job takes as long as its slowest rank (all-reduce MAX; identity on one rank)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(step_flops: float, ms_per_step: float, world: int) -> float:
+    """Selected-pair TFLOP/s of the whole job: every rank did step_flops in ms_per_step."""
+    return world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+
 # ---- our arm -----------------------------------------------------------------------------------
 def time_region(fn, reps, stream):
     """Median CUDA-event time (ms) of fn() over reps runs."""
@@ -257,7 +277,7 @@ def run_ours(args):
     # eight independent layers' inputs: host (pinned) and device copies
     host = []
     for layer in range(LAYERS):
-        host.append(tuple(t.pin_memory() for t in I.draw_qkv(w, layer=layer + rank * LAYERS)))
+        host.append(tuple(t.pin_memory() for t in I.draw_qkv(w, layer=rank_layer_seed_offset(rank, layer))))
     devb = [tuple(t.to(dev) for t in h) for h in host]
     outs = [torch.empty((T, w.hq, w.d), dtype=torch.bfloat16, device=dev) for _ in range(LAYERS)]
     lses = [torch.empty((w.hq, T), dtype=torch.float32, device=dev) for _ in range(LAYERS)]
@@ -301,12 +321,9 @@ def run_ours(args):
     total_ms = e0.elapsed_time(e1)
     route.check_status()
     assert int(route.total_pairs.item()) == pairs
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_value(step_flops, ms_per_step, world)
     kern_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_ms) / LAYERS
 
     # ---- end to end: pinned host buffers -> device -> kernels -> host, every step
@@ -334,11 +351,8 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * step_flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    e2e_value = whole_job_value(step_flops, e2e_ms / e2e_steps, world)
 
     if rank != 0:
         if dist is not None:
