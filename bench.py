@@ -361,11 +361,13 @@ def run_ours(args):
 
     peaks = measured_peaks()
     achieved = layer_flops / (kern_ms * 1e-3) / 1e12
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "attn_fwd_qwen_32k_traffic.json")
+    traffic = None   # dram__bytes_read + dram__bytes_write per launch, from the committed ncu summary
+    tpath = os.path.join(ROOT, "profiles", "attn_fwd_kernel_qwen_32k.md")
     if os.path.exists(tpath):
+        import re
         with open(tpath) as f:
-            traffic = json.load(f).get("dram_bytes_per_launch")
+            m = re.search(r"^dram_bytes_per_launch\s*=\s*(\d+)", f.read(), re.M)
+        traffic = int(m.group(1)) if m else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
