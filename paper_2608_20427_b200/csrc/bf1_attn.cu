@@ -94,7 +94,9 @@ struct Cfg {
     static constexpr int kRing = (D == 128) ? 4 : 8;       // ring slots
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = kQBytes;
-    static constexpr int kHandOff = kRingOff + kRing * kTileBytes;          // Handoff[2]
+    static constexpr int kStageOff = kRingOff + kRing * kTileBytes;         // O staging: 4 warps x 32 rows x 64 B
+    static constexpr int kStageBytes = 4 * 32 * 64;
+    static constexpr int kHandOff = kStageOff + kStageBytes;                // Handoff[2]
     static constexpr int kQueueOff = kHandOff + 2 * (int)sizeof(Handoff);   // QueueEntry[kQueue]
     static constexpr int kInfoOff = kQueueOff + kQueue * (int)sizeof(QueueEntry);   // int4[2]
     static constexpr int kBarOff = kInfoOff + 32;
@@ -187,6 +189,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k,
                                                                const __grid_constant__ CUtensorMap tm_v,
+                                                               const __grid_constant__ CUtensorMap tm_o,
                                                                const AttnArgs args) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -273,6 +276,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
     }
     __syncwarp();
     if (warp == 1) {
@@ -365,50 +369,56 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     __syncwarp();
                     if (++slot == C::kRing) { slot = 0; ++pass; }
                 };
-                // K0 only needs a ring slot, not the Q buffer: get it going first
-                int p_prev = __shfl_sync(0xffffffffu, my_p, 0);
-                if (cnt > 0) load_tile(p_prev, false);
-                if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
-                TR(tr, 1, n);
-                if (elect_one()) {
-                    // publish the unit (or the end marker cnt = 0) to the MMA and softmax warps
-                    s_info[n & 1].x = cnt;
-                    s_info[n & 1].y = rows_valid;
-                    s_info[n & 1].z = tok0;
-                    s_info[n & 1].w = kvh;
-                    mbar_arrive(bar_info + 8 * (n & 1));
-                    if (cnt == 0) {
-                        mbar_arrive(bar_q_full);
-                    } else {
-                        mbar_expect_tx(bar_q_full, C::kQBytes);
-                        // one copy: box = 64 elements x 64 tokens x 2 heads x all column chunks
-                        tma_load_4d(sQ, &tm_q, 0, tok0, kvh * 2, 0, bar_q_full);
-                    }
-                }
-                __syncwarp();
-                if (cnt == 0) break;
-                // K1, V0, K2, V1, ...: the order in which the MMA warp consumes them
+                // One loop body for every step keeps the producer's code small and hot in the
+                // instruction cache.  Step s loads K(s) and then V(s-1): K0, [Q], K1, V0, K2, V1, ...,
+                // the order in which the MMA warp consumes them.  K0 only needs a ring slot, so it
+                // is started before the wait for the Q buffer.
                 int base_i = 0;
-                for (int i = 1; i < cnt; ++i) {
-                    if (i - base_i == 32) {   // lists longer than a warp: fetch the next 32 entries
-                        base_i += 32;
-                        const int ii = base_i + lane;
-                        int p = 0;
-                        if (ii < cnt) {
-                            p = args.dense ? ii : args.kv_idx[(size_t)rslot * args.max_degree + ii];
-                            if (p < 0 || p > j || (ii == cnt - 1) != (p == j)) {
-                                if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
-                                p = (ii == cnt - 1) ? j : 0;
+                int p_prev = 0;
+                for (int st = 0; st <= cnt; ++st) {
+                    int p_cur = 0;
+                    if (st < cnt) {
+                        if (st - base_i == 32) {   // lists longer than a warp: fetch the next 32 entries
+                            base_i += 32;
+                            const int ii = base_i + lane;
+                            int p = 0;
+                            if (ii < cnt) {
+                                p = args.dense ? ii : args.kv_idx[(size_t)rslot * args.max_degree + ii];
+                                if (p < 0 || p > j || (ii == cnt - 1) != (p == j)) {
+                                    if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
+                                    p = (ii == cnt - 1) ? j : 0;
+                                }
+                            }
+                            my_p = p;
+                        }
+                        p_cur = __shfl_sync(0xffffffffu, my_p, st - base_i);
+                        load_tile(p_cur, false);
+                    }
+                    if (st == 0) {
+                        if (n > 0) mbar_wait(bar_q_free, (n - 1) & 1, abort_flag, args.status);
+                        TR(tr, 1, n);
+                        if (elect_one()) {
+                            // publish the unit (or the end marker cnt = 0) to the MMA and softmax warps
+                            s_info[n & 1].x = cnt;
+                            s_info[n & 1].y = rows_valid;
+                            s_info[n & 1].z = tok0;
+                            s_info[n & 1].w = kvh;
+                            mbar_arrive(bar_info + 8 * (n & 1));
+                            if (cnt == 0) {
+                                mbar_arrive(bar_q_full);
+                            } else {
+                                mbar_expect_tx(bar_q_full, C::kQBytes);
+                                // one copy: box = 64 elements x 64 tokens x 2 heads x all column chunks
+                                tma_load_4d(sQ, &tm_q, 0, tok0, kvh * 2, 0, bar_q_full);
                             }
                         }
-                        my_p = p;
+                        __syncwarp();
+                    } else {
+                        load_tile(p_prev, true);
                     }
-                    const int p_cur = __shfl_sync(0xffffffffu, my_p, i - base_i);
-                    load_tile(p_cur, false);
-                    load_tile(p_prev, true);
                     p_prev = p_cur;
                 }
-                load_tile(p_prev, true);
+                if (cnt == 0) break;
                 if (elect_one()) mbar_arrive(bar_sq_free + 8 * qs);
                 __syncwarp();
                 TR(tr, 3, n);
@@ -473,39 +483,42 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 const int cnt = s_info[n & 1].x;
                 TR(tr, 14, n);
                 if (cnt == 0 || *abort_flag) break;
-                issue_s(g);
-                if (cnt == 1 && elect_one()) mma_commit(bar_q_free);
-                __syncwarp();
-                for (int i = 0; i < cnt; ++i, ++g) {
-                    if (i + 1 < cnt) {
-                        issue_s(g + 1);
+                // One loop body for every step (small, hot in the instruction cache): step s issues
+                // S(s) and then PV(s-1), i.e. S0, S1, PV0, S2, PV1, ..., PV(cnt-1).
+                for (int st = 0; st <= cnt; ++st) {
+                    if (st < cnt) {
+                        issue_s(g + st);
                         // last S of the unit: Q may be replaced
-                        if (i + 2 == cnt && elect_one()) mma_commit(bar_q_free);
+                        if (st == cnt - 1 && elect_one()) mma_commit(bar_q_free);
                         __syncwarp();
                     }
-                    mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);           // V(i) landed
-                    TR(tr, 11, g);
-                    mbar_wait(bar_p_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);  // P(i) written
-                    TR(tr, 12, g);
-                    if (i == 0 && n > 0) mbar_wait(bar_o_free, (n - 1) & 1, abort_flag, args.status);
-                    TR(tr, 13, g);
-                    tc_fence_after();
-                    // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
-                    // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
-                    const uint32_t v_lo = v_lo0 + slot * (C::kTileBytes >> 4);
-                    const uint32_t a_p = tmem + C::kColS + (g & 1) * 64;
-                    if (elect_one()) {
-                        if (i == 0) mma_ts_lohi<false>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
-                        else mma_ts_lohi<true>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
+                    if (st >= 1) {
+                        const uint32_t gi = g + st - 1;
+                        mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);             // V landed
+                        TR(tr, 11, gi);
+                        mbar_wait(bar_p_full + 8 * (gi & 1), (gi >> 1) & 1, abort_flag, args.status);  // P written
+                        TR(tr, 12, gi);
+                        if (st == 1 && n > 0) mbar_wait(bar_o_free, (n - 1) & 1, abort_flag, args.status);
+                        TR(tr, 13, gi);
+                        tc_fence_after();
+                        // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
+                        // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
+                        const uint32_t v_lo = v_lo0 + slot * (C::kTileBytes >> 4);
+                        const uint32_t a_p = tmem + C::kColS + (gi & 1) * 64;
+                        if (elect_one()) {
+                            if (st == 1) mma_ts_lohi<false>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
+                            else mma_ts_lohi<true>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
 #pragma unroll
-                        for (int kk = 1; kk < kBlock / 16; ++kk)
-                            mma_ts_lohi<true>(tmem + C::kColO, a_p + kk * 8, v_lo + kk * (2048 >> 4), kDescHi, kIdescO);
-                        mma_commit(bar_free + 8 * slot);
-                        mma_commit(bar_pv_done + 8 * (g & 1));
+                            for (int kk = 1; kk < kBlock / 16; ++kk)
+                                mma_ts_lohi<true>(tmem + C::kColO, a_p + kk * 8, v_lo + kk * (2048 >> 4), kDescHi, kIdescO);
+                            mma_commit(bar_free + 8 * slot);
+                            mma_commit(bar_pv_done + 8 * (gi & 1));
+                        }
+                        __syncwarp();
+                        if (++slot == C::kRing) { slot = 0; ++pass; }
                     }
-                    __syncwarp();
-                    if (++slot == C::kRing) { slot = 0; ++pass; }
                 }
+                g += cnt;
             }
 #ifdef BF1_TRACE
             if (lane == 0) *(volatile int*)(s_nqb + 1) = 1;   // tells the trace probe to stop
@@ -644,9 +657,20 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             const int tok = tok0 + tl;
             const bool store = tl < rows_valid;
             __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * 2 + hl)) * D;
-            // 16 columns at a time keeps this warpgroup inside its small register budget
+            // Full blocks leave through shared memory and TMA stores: each warp packs 32 rows x 32
+            // columns into its own 2 KB staging tile (64-byte swizzle, conflict-free) and one lane
+            // hands it to the copy engine.  Scattered 16-byte global stores from here would sit in the
+            // same load/store path as every other warp's mbarrier and shared-memory traffic and
+            // slow the whole SM down.  16 columns at a time keeps the register budget small.
+            const bool full_tile = rows_valid == kBlock;   // warp-uniform
+            const uint32_t stage_w = base + C::kStageOff + (warp & 3) * 2048;
+            const uint32_t srow = stage_w + lane * 64;
 #pragma unroll
             for (int c = 0; c < D / 16; ++c) {
+                if (full_tile && (c & 1) == 0) {
+                    if (lane == 0) bulk_wait_read0();   // the previous store has finished reading the tile
+                    __syncwarp();
+                }
                 uint32_t oreg[16];
                 tmem_ld16(t_lane + C::kColO + c * 16, oreg);
                 tmem_wait_ld();
@@ -655,16 +679,30 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_o_free);
                 }
-                if (store) {
-                    uint4 w0, w1;
-                    w0.x = pack_bf16x2(__uint_as_float(oreg[0]) * inv_l, __uint_as_float(oreg[1]) * inv_l);
-                    w0.y = pack_bf16x2(__uint_as_float(oreg[2]) * inv_l, __uint_as_float(oreg[3]) * inv_l);
-                    w0.z = pack_bf16x2(__uint_as_float(oreg[4]) * inv_l, __uint_as_float(oreg[5]) * inv_l);
-                    w0.w = pack_bf16x2(__uint_as_float(oreg[6]) * inv_l, __uint_as_float(oreg[7]) * inv_l);
-                    w1.x = pack_bf16x2(__uint_as_float(oreg[8]) * inv_l, __uint_as_float(oreg[9]) * inv_l);
-                    w1.y = pack_bf16x2(__uint_as_float(oreg[10]) * inv_l, __uint_as_float(oreg[11]) * inv_l);
-                    w1.z = pack_bf16x2(__uint_as_float(oreg[12]) * inv_l, __uint_as_float(oreg[13]) * inv_l);
-                    w1.w = pack_bf16x2(__uint_as_float(oreg[14]) * inv_l, __uint_as_float(oreg[15]) * inv_l);
+                uint4 w0, w1;
+                w0.x = pack_bf16x2(__uint_as_float(oreg[0]) * inv_l, __uint_as_float(oreg[1]) * inv_l);
+                w0.y = pack_bf16x2(__uint_as_float(oreg[2]) * inv_l, __uint_as_float(oreg[3]) * inv_l);
+                w0.z = pack_bf16x2(__uint_as_float(oreg[4]) * inv_l, __uint_as_float(oreg[5]) * inv_l);
+                w0.w = pack_bf16x2(__uint_as_float(oreg[6]) * inv_l, __uint_as_float(oreg[7]) * inv_l);
+                w1.x = pack_bf16x2(__uint_as_float(oreg[8]) * inv_l, __uint_as_float(oreg[9]) * inv_l);
+                w1.y = pack_bf16x2(__uint_as_float(oreg[10]) * inv_l, __uint_as_float(oreg[11]) * inv_l);
+                w1.z = pack_bf16x2(__uint_as_float(oreg[12]) * inv_l, __uint_as_float(oreg[13]) * inv_l);
+                w1.w = pack_bf16x2(__uint_as_float(oreg[14]) * inv_l, __uint_as_float(oreg[15]) * inv_l);
+                if (full_tile) {
+                    const int ch = (c & 1) * 2;           // 16-byte chunk inside the 64-byte staging row
+                    const int sw = (lane >> 1) & 3;       // 64-byte swizzle: chunk ^= (row / 2) % 4
+                    st_shared_v4(srow + (((ch + 0) ^ sw) << 4), w0.x, w0.y, w0.z, w0.w);
+                    st_shared_v4(srow + (((ch + 1) ^ sw) << 4), w1.x, w1.y, w1.z, w1.w);
+                    if (c & 1) {
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_3d(&tm_o, (c >> 1) * 32, kvh * 2 + hl, tok0 + (quarter & 1) * 32, stage_w);
+                            bulk_commit_group();
+                        }
+                    }
+                } else if (store) {
+                    // partial last block of a sequence: the rows after it belong to someone else
                     *reinterpret_cast<uint4*>(orow + c * 16) = w0;
                     *reinterpret_cast<uint4*>(orow + c * 16 + 8) = w1;
                 }
@@ -676,6 +714,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         }
     }
 
+    if (warp >= 8 && lane == 0) bulk_wait0();   // this thread's output stores have landed
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
@@ -717,6 +756,22 @@ static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, in
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(BF1_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return BF1_OK;
+}
+
+// O [T, Hq, d] bf16 for the epilogue's TMA stores: box = 32 elements (64 bytes) x 1 head x 32 tokens,
+// 64-byte swizzle.
+static int make_store_map(CUtensorMap* m, void* ptr, int64_t T, int H, int d) {
+    EncodeTiledFn enc;
+    if (int rc = get_encode_fn(&enc)) return rc;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)T};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)H * d * 2};
+    cuuint32_t box[3] = {32, 1, 32};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptr, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(BF1_ERR_CUDA, "cuTensorMapEncodeTiled (O) failed with CUresult %d", (int)r);
     return BF1_OK;
 }
 
@@ -778,7 +833,8 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     DeviceInfo info;
     if (int rc = device_info(&info)) return rc;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
+    if (int rc = make_store_map(&to, o, total_tokens, hq, d)) return rc;
     if (int rc = make_map(&tq, q, total_tokens, hq, d, 2)) return rc;
     if (int rc = make_map(&tk, k, total_tokens, hkv, d, 1)) return rc;
     if (int rc = make_map(&tv, v, total_tokens, hkv, d, 1)) return rc;
@@ -808,9 +864,9 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     const int64_t units = slots * hkv;
     const int grid = (int)(units < 2LL * info.sm_count ? units : 2LL * info.sm_count);
     if (d == 128)
-        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
+        attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);
     else
-        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, a);
+        attn_fwd_kernel<64><<<grid, kThreads, Cfg<64>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
 }
