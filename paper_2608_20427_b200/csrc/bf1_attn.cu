@@ -238,6 +238,15 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     int* s_abort = reinterpret_cast<int*>(smem + C::kMiscOff + 4);
     int* s_nqb = reinterpret_cast<int*>(smem + C::kMiscOff + 8);
 
+#ifdef BF1_TRACE
+    Tracer tr_cta;
+    if (tid == 32) {   // lane 0 of the MMA warp: shares that role's trace area
+        tr_cta.init(1);
+        tr_cta.p = tr_cta.p ? tr_cta.p + 2 * (tr_cta.cap - 8) : nullptr;   // last 8 records
+        tr_cta.cap = 8;
+        TR(tr_cta, 40, 0);
+    }
+#endif
     if (tid == 0) {
         *s_abort = 0;
         if (base & 1023u) {   // the swizzled tiles need a 1024-byte aligned window
@@ -290,6 +299,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     volatile int* abort_flag = s_abort;
     const int nqb = *s_nqb;
     const int total_units = nqb * args.hkv;
+#ifdef BF1_TRACE
+    if (tid == 32) TR(tr_cta, 41, 0);
+#endif
 
     if (warp < 4) {
         setmaxnreg_dec<kRegsCtl>();
@@ -451,6 +463,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             uint32_t g = 0;   // tiles issued so far by this CTA; S buffer = g & 1
             Tracer tr;
             if (lane == 0) tr.init(1);
+#ifdef BF1_TRACE
+            tr.cap = tr.cap > 8 ? tr.cap - 8 : 0;   // the last records belong to the CTA-level marks
+#endif
             // Descriptor halves that never change: the high word (SBO = 1024, version, swizzle) and
             // the low words of Q's eight k-slices; a ring slot only adds slot * kTileBytes / 16.
             constexpr uint32_t kDescHi = desc_hi_sw128(1024);
@@ -717,6 +732,9 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     if (warp >= 8 && lane == 0) bulk_wait0();   // this thread's output stores have landed
     tc_fence_before();
     __syncthreads();
+#ifdef BF1_TRACE
+    if (tid == 32) TR(tr_cta, 42, 0);
+#endif
     if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
     retire();
 }
