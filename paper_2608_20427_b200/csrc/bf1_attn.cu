@@ -18,8 +18,9 @@
 // register budgets are re-balanced with setmaxnreg:
 //   warp 0      TMA producer: Q once per unit, then K and V tiles through a ring of 16 KB slots
 //               in the order the MMAs consume them (K0, K1, V0, K2, V1, ...),
-//   warp 1      MMA issuer: S(g+1) is issued before PV(g), so the tensor pipe works on the next
-//               tile's scores and the previous tile's PV while the softmax warps are busy,
+//   warp 1      MMA issuer for S = Q K^T: runs up to two tiles ahead of the softmax (two S buffers),
+//   warp 3      MMA issuer for O += P V: a separate warp, so that neither kind of MMA waits behind
+//               a burst of the other while the tensor pipe's queue is full,
 //   warp 2      scheduler: fetches the next unit, decodes it, reads (and range-checks) its list,
 //               prefetches its Q/K/V blocks into L2 and queues it for the producer -- all of it
 //               global-memory latency that must not sit in front of the copies,
@@ -355,9 +356,6 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             int slot = 0, pass = 0;
             Tracer tr;
             if (lane == 0) tr.init(0);
-#ifdef BF1_TRACE
-            tr.cap = tr.cap / 2;   // the second half is the landing probe's
-#endif
             int n_tiles = 0;
             (void)n_tiles;
             for (int n = 0;; ++n) {
@@ -435,109 +433,108 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 __syncwarp();
                 TR(tr, 3, n);
             }
-#ifdef BF1_TRACE
-        } else if (warp == 3) {
-            // trace builds only: watch the ring's "full" barriers and record when each copy lands
-            if (lane == 0) {
-                Tracer tr;
-                tr.init(0);
-                tr.p = tr.p ? tr.p + 2 * (tr.cap / 2) : nullptr;   // second half of the producer's trace area
-                tr.cap = tr.cap / 2;
-                int slot = 0, pass = 0;
-                for (int e = 0;; ++e) {
-                    bool ok = false;
-                    while (!(ok = mbar_try_wait(bar_full + 8 * slot, pass & 1)) && !*(volatile int*)(s_nqb + 1)) {}
-                    if (!ok) break;
-                    TR(tr, 30, e);
-                    if (++slot == C::kRing) { slot = 0; ++pass; }
-                }
-            }
-#endif
         } else if (warp == 1) {
-            // ================================ MMA issuer ======================================
+            // ================================ MMA issuer: S = Q K^T ============================
             // The whole warp walks the loop (so that addresses and descriptors stay warp-uniform and
-            // cheap); one elected lane issues the MMAs and commits.
+            // cheap); one elected lane issues the MMAs and commits.  S and PV have separate issuing
+            // warps: an issuer stalls while the tensor pipe's queue is full, and with one issuer a
+            // stalled burst of S MMAs would keep a ready PV (which frees an S buffer and feeds the
+            // epilogue) waiting behind it, and the other way round.
             constexpr uint32_t kIdescS = idesc_bf16_f32(kBlock, false);   // 128 x 64 x 16, K-major B
-            constexpr uint32_t kIdescO = idesc_bf16_f32(D, true);         // 128 x D x 16, MN-major B
-            int slot = 0, pass = 0, n = 0;
-            uint32_t g = 0;   // tiles issued so far by this CTA; S buffer = g & 1
+            static_assert((C::kRing & (C::kRing - 1)) == 0, "ring size must be a power of two");
+            uint32_t g = 0;    // tiles before this unit; S buffer of tile t = t & 1
+            uint32_t e0 = 0;   // ring fills before this unit
             Tracer tr;
             if (lane == 0) tr.init(1);
 #ifdef BF1_TRACE
-            tr.cap = tr.cap > 8 ? tr.cap - 8 : 0;   // the last records belong to the CTA-level marks
+            tr.cap = tr.cap / 2;   // the second half belongs to the PV issuer and the CTA-level marks
 #endif
             // Descriptor halves that never change: the high word (SBO = 1024, version, swizzle) and
             // the low words of Q's eight k-slices; a ring slot only adds slot * kTileBytes / 16.
             constexpr uint32_t kDescHi = desc_hi_sw128(1024);
             const uint32_t q_lo = desc_lo_sw128(sQ, 16);
             const uint32_t k_lo0 = desc_lo_sw128(sRing, 16);
-            const uint32_t v_lo0 = desc_lo_sw128(sRing, kBlock * 128);
-            auto issue_s = [&](uint32_t gt) {
-                TR(tr, 9, gt);
-                mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);
-                TR(tr, 10, gt);
-                tc_fence_after();
-                const uint32_t k_lo = k_lo0 + slot * (C::kTileBytes >> 4);
-                const uint32_t d_s = tmem + C::kColS + (gt & 1) * 64;
-                if (elect_one()) {
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t a_off = ((kk / 4) * (kRows * 128) + (kk % 4) * 32) >> 4;
-                        const uint32_t b_off = ((kk / 4) * (kBlock * 128) + (kk % 4) * 32) >> 4;
-                        if (kk == 0) mma_ss_lohi<false>(d_s, q_lo + a_off, k_lo + b_off, kDescHi, kIdescS);
-                        else mma_ss_lohi<true>(d_s, q_lo + a_off, k_lo + b_off, kDescHi, kIdescS);
-                    }
-                    mma_commit(bar_free + 8 * slot);
-                    mma_commit(bar_s_full + 8 * (gt & 1));
-                }
-                __syncwarp();
-                if (++slot == C::kRing) { slot = 0; ++pass; }
-            };
-            for (;; ++n) {
+            for (int n = 0;; ++n) {
                 mbar_wait(bar_q_full, n & 1, abort_flag, args.status);
                 const int cnt = s_info[n & 1].x;
                 TR(tr, 14, n);
                 if (cnt == 0 || *abort_flag) break;
-                // One loop body for every step (small, hot in the instruction cache): step s issues
-                // S(s) and then PV(s-1), i.e. S0, S1, PV0, S2, PV1, ..., PV(cnt-1).
-                for (int st = 0; st <= cnt; ++st) {
-                    if (st < cnt) {
-                        issue_s(g + st);
-                        // last S of the unit: Q may be replaced
-                        if (st == cnt - 1 && elect_one()) mma_commit(bar_q_free);
-                        __syncwarp();
-                    }
-                    if (st >= 1) {
-                        const uint32_t gi = g + st - 1;
-                        mbar_wait(bar_full + 8 * slot, pass & 1, abort_flag, args.status);             // V landed
-                        TR(tr, 11, gi);
-                        mbar_wait(bar_p_full + 8 * (gi & 1), (gi >> 1) & 1, abort_flag, args.status);  // P written
-                        TR(tr, 12, gi);
-                        if (st == 1 && n > 0) mbar_wait(bar_o_free, (n - 1) & 1, abort_flag, args.status);
-                        TR(tr, 13, gi);
-                        tc_fence_after();
-                        // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
-                        // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
-                        const uint32_t v_lo = v_lo0 + slot * (C::kTileBytes >> 4);
-                        const uint32_t a_p = tmem + C::kColS + (gi & 1) * 64;
-                        if (elect_one()) {
-                            if (st == 1) mma_ts_lohi<false>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
-                            else mma_ts_lohi<true>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
+                for (int st = 0; st < cnt; ++st) {
+                    const uint32_t t = g + st;
+                    const uint32_t e = e0 + (st == 0 ? 0 : 2 * st - 1);   // ring fill holding K(st): K0, K1, V0, K2, V1, ...
+                    const uint32_t slot = e & (C::kRing - 1);
+                    TR(tr, 9, t);
+                    mbar_wait(bar_full + 8 * slot, (e / C::kRing) & 1, abort_flag, args.status);   // K landed
+                    // S(t) overwrites the buffer that held P(t-2): PV(t-2) must have finished with it
+                    if (t >= 2) mbar_wait(bar_pv_done + 8 * (t & 1), ((t - 2) >> 1) & 1, abort_flag, args.status);
+                    TR(tr, 10, t);
+                    tc_fence_after();
+                    const uint32_t k_lo = k_lo0 + slot * (C::kTileBytes >> 4);
+                    const uint32_t d_s = tmem + C::kColS + (t & 1) * 64;
+                    if (elect_one()) {
 #pragma unroll
-                            for (int kk = 1; kk < kBlock / 16; ++kk)
-                                mma_ts_lohi<true>(tmem + C::kColO, a_p + kk * 8, v_lo + kk * (2048 >> 4), kDescHi, kIdescO);
-                            mma_commit(bar_free + 8 * slot);
-                            mma_commit(bar_pv_done + 8 * (gi & 1));
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t a_off = ((kk / 4) * (kRows * 128) + (kk % 4) * 32) >> 4;
+                            const uint32_t b_off = ((kk / 4) * (kBlock * 128) + (kk % 4) * 32) >> 4;
+                            if (kk == 0) mma_ss_lohi<false>(d_s, q_lo + a_off, k_lo + b_off, kDescHi, kIdescS);
+                            else mma_ss_lohi<true>(d_s, q_lo + a_off, k_lo + b_off, kDescHi, kIdescS);
                         }
-                        __syncwarp();
-                        if (++slot == C::kRing) { slot = 0; ++pass; }
+                        mma_commit(bar_free + 8 * slot);
+                        mma_commit(bar_s_full + 8 * (t & 1));
+                        if (st == cnt - 1) mma_commit(bar_q_free);   // last S of the unit: Q may be replaced
                     }
+                    __syncwarp();
                 }
                 g += cnt;
+                e0 += 2 * cnt;
             }
+        } else if (warp == 3) {
+            // ================================ MMA issuer: O += P V =============================
+            constexpr uint32_t kIdescO = idesc_bf16_f32(D, true);         // 128 x D x 16, MN-major B
+            constexpr uint32_t kDescHi = desc_hi_sw128(1024);
+            const uint32_t v_lo0 = desc_lo_sw128(sRing, kBlock * 128);
+            uint32_t g = 0, e0 = 0;
+            Tracer tr;
 #ifdef BF1_TRACE
-            if (lane == 0) *(volatile int*)(s_nqb + 1) = 1;   // tells the trace probe to stop
+            if (lane == 0) {   // second half of the S issuer's trace area
+                tr.init(1);
+                tr.p = tr.p ? tr.p + 2 * (tr.cap / 2) : nullptr;
+                tr.cap = tr.cap / 2 - 8;
+            }
 #endif
+            for (int n = 0;; ++n) {
+                mbar_wait(bar_info + 8 * (n & 1), (n >> 1) & 1, abort_flag, args.status);
+                const int cnt = s_info[n & 1].x;
+                if (cnt == 0 || *abort_flag) break;
+                for (int st = 0; st < cnt; ++st) {
+                    const uint32_t t = g + st;
+                    const uint32_t e = e0 + (st == cnt - 1 ? 2 * cnt - 1 : 2 * st + 2);   // ring fill holding V(st)
+                    const uint32_t slot = e & (C::kRing - 1);
+                    mbar_wait(bar_full + 8 * slot, (e / C::kRing) & 1, abort_flag, args.status);       // V landed
+                    TR(tr, 11, t);
+                    mbar_wait(bar_p_full + 8 * (t & 1), (t >> 1) & 1, abort_flag, args.status);        // P written
+                    TR(tr, 12, t);
+                    if (st == 0 && n > 0) mbar_wait(bar_o_free, (n - 1) & 1, abort_flag, args.status);
+                    TR(tr, 13, t);
+                    tc_fence_after();
+                    // V tile: rows = kv tokens (the K of this MMA), 128-byte rows of 64 d-elements;
+                    // 16 kv rows per MMA = two 8-row groups = 2048 bytes; next d chunk 8 KB away
+                    const uint32_t v_lo = v_lo0 + slot * (C::kTileBytes >> 4);
+                    const uint32_t a_p = tmem + C::kColS + (t & 1) * 64;
+                    if (elect_one()) {
+                        if (st == 0) mma_ts_lohi<false>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
+                        else mma_ts_lohi<true>(tmem + C::kColO, a_p, v_lo, kDescHi, kIdescO);
+#pragma unroll
+                        for (int kk = 1; kk < kBlock / 16; ++kk)
+                            mma_ts_lohi<true>(tmem + C::kColO, a_p + kk * 8, v_lo + kk * (2048 >> 4), kDescHi, kIdescO);
+                        mma_commit(bar_free + 8 * slot);
+                        mma_commit(bar_pv_done + 8 * (t & 1));
+                    }
+                    __syncwarp();
+                }
+                g += cnt;
+                e0 += 2 * cnt;
+            }
         }
         __syncwarp();
     } else if (warp < 8) {
