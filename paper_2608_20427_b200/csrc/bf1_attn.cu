@@ -495,6 +495,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             const uint32_t v_lo0 = desc_lo_sw128(sRing, kBlock * 128);
             uint32_t g = 0, e0 = 0;
             Tracer tr;
+            (void)tr;
 #ifdef BF1_TRACE
             if (lane == 0) {   // second half of the S issuer's trace area
                 tr.init(1);

@@ -12,7 +12,6 @@
 namespace bf1 {
 
 // ---- host: thread-local error string ------------------------------------------------
-void set_error(const char* fmt, ...);
 int fail(int code, const char* fmt, ...);
 
 #define BF1_CUDA_CHECK(expr)                                                              \
