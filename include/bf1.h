@@ -166,6 +166,49 @@ int bf1_attn_fwd_noalloc(const void *q, const void *k, const void *v, const int3
                          const bf1_route_cfg *cfg /* host */, void *o, float *lse,
                          int32_t *status_dev, void *stream);
 
+/* ---- cached one-token decode over selected KV pages (Section 3.2, Section 5.4) -----------------
+ * The newest token of a sequence with n cached tokens (position n-1, block j = (n-1)/64) attends to
+ * the pages of P(j), the self page only up to token n-1: O(log B) pages per step.  The KV cache is
+ * paged: k_pages / v_pages are [num_pages, 64, hkv, d] bf16 and page_table[s, i] names the
+ * physical page that holds logical block i of sequence s.  The page list changes only when n
+ * crosses a block boundary, so one plan serves a whole 64-token route epoch (the paper's open
+ * item: "persistent plan reuse across a 64-token route epoch"). */
+typedef struct {
+    int32_t  max_degree;   /* host: row pitch of `page`                                          */
+    int32_t *count;        /* [batch] pages to read for the sequence (0 for an empty sequence)   */
+    int32_t *page;         /* [batch, max_degree] physical pages in ascending logical-block
+                              order, the self page last; unused entries = -1                     */
+    int32_t *block;        /* [batch] block index j the plan was made for (-1 if empty)          */
+    int32_t *status;       /* [1] BF1_DEV_* bits; written by bf1_plan_decode, OR-ed by the
+                              attention call                                                     */
+} bf1_decode_plan;         /* all pointers: device memory owned by the caller                    */
+
+/* Eq. 1 for the newest token's block of every sequence, mapped through the page table.
+ *   seqlens_dev     [batch] int32 device: cached tokens per sequence (0 allowed)
+ *   page_table_dev  [batch, max_pages_per_seq] int32 device
+ * A sequence that needs a logical block >= max_pages_per_seq sets BF1_DEV_BAD_SEQLENS. */
+int bf1_plan_decode(const int32_t *seqlens_dev, const int32_t *page_table_dev,
+                    int32_t max_pages_per_seq, int32_t batch, const bf1_route_cfg *cfg /* host */,
+                    const bf1_decode_plan *out /* host struct, device arrays */, void *stream);
+
+/* Bytes of device scratch bf1_decode_fwd needs (partial results of the split over pages and one
+ * ticket word per sequence and KV head).  Host only; -1 on bad arguments. */
+int64_t bf1_decode_workspace_bytes(int32_t batch, int32_t hkv, int32_t max_degree, int32_t d);
+
+/* One decode step for every sequence of the batch.
+ *   q            device bf16 [batch, hq, d]: the newest token's queries
+ *   seqlens_dev  [batch] current cached lengths INCLUDING the newest token; must lie in the block
+ *                the plan was made for, otherwise BF1_DEV_BAD_ROUTE is set and the sequence skipped
+ *   workspace    device, 16-byte aligned, bf1_decode_workspace_bytes() bytes, all zero before the
+ *                first call; every call leaves its ticket words at zero again, so it can be
+ *                reused by calls that do not overlap on the GPU
+ *   o            device bf16 [batch, hq, d];  lse  device fp32 [hq, batch]
+ * Rows of empty sequences are not written.  Geometry limits as for bf1_attn_fwd. */
+int bf1_decode_fwd(const void *q, const void *k_pages, const void *v_pages, int32_t num_pages,
+                   const int32_t *seqlens_dev, int32_t batch, int32_t hq, int32_t hkv, int32_t d,
+                   float softmax_scale, const bf1_decode_plan *plan /* host */, void *workspace,
+                   void *o, float *lse, void *stream);
+
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char *bf1_last_error(void);
 

@@ -19,7 +19,8 @@ BF1_OK = 0
 DEV_BAD_SEQLENS, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_ROUTE = 1, 2, 4, 8
 
 EXPORTS = ("bf1_route_capacity", "bf1_plan_route", "bf1_attn_fwd", "bf1_dense_causal_fwd",
-           "bf1_attn_fwd_noalloc", "bf1_last_error", "bf1_version")
+           "bf1_attn_fwd_noalloc", "bf1_plan_decode", "bf1_decode_workspace_bytes", "bf1_decode_fwd",
+           "bf1_last_error", "bf1_version")
 
 
 class RouteCfg(ctypes.Structure):
@@ -39,6 +40,12 @@ class _RouteC(ctypes.Structure):
                 ("pair_count", ctypes.c_void_p), ("order", ctypes.c_void_p),
                 ("total_pairs", ctypes.c_void_p), ("num_qblocks", ctypes.c_void_p),
                 ("status", ctypes.c_void_p), ("sched", ctypes.c_void_p)]
+
+
+class _DecodePlanC(ctypes.Structure):
+    """Mirror of bf1_decode_plan."""
+    _fields_ = [("max_degree", ctypes.c_int32), ("count", ctypes.c_void_p), ("page", ctypes.c_void_p),
+                ("block", ctypes.c_void_p), ("status", ctypes.c_void_p)]
 
 
 class Bf1Error(RuntimeError):
@@ -69,6 +76,13 @@ def load():
     L.bf1_attn_fwd_noalloc.restype = ctypes.c_int
     L.bf1_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(RouteCfg),
                                        vp, vp, vp, vp]
+    L.bf1_plan_decode.restype = ctypes.c_int
+    L.bf1_plan_decode.argtypes = [vp, vp, i32, i32, ctypes.POINTER(RouteCfg), ctypes.POINTER(_DecodePlanC), vp]
+    L.bf1_decode_workspace_bytes.restype = i64
+    L.bf1_decode_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.bf1_decode_fwd.restype = ctypes.c_int
+    L.bf1_decode_fwd.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, f32, ctypes.POINTER(_DecodePlanC), vp, vp,
+                                 vp, vp]
     L.bf1_last_error.restype = ctypes.c_char_p
     L.bf1_last_error.argtypes = []
     L.bf1_version.restype = ctypes.c_int
@@ -210,6 +224,61 @@ def attn_fwd_noalloc(q, k, v, cu_seqlens, max_seqlen: int, out, lse, cfg: Option
                                        float(scale) if scale else 0.0, ctypes.byref(cfg), out.data_ptr(),
                                        lse.data_ptr(), status.data_ptr() if status is not None else None,
                                        _stream_ptr(stream)))
+    return out, lse
+
+
+@dataclass
+class DecodePlan:
+    """Device arrays of a decode plan (one page list per sequence) plus the C struct."""
+    max_degree: int
+    count: torch.Tensor
+    page: torch.Tensor
+    block: torch.Tensor
+    status: torch.Tensor
+    c: _DecodePlanC = None
+
+    @staticmethod
+    def empty(batch: int, max_degree: int, device) -> "DecodePlan":
+        i32 = dict(dtype=torch.int32, device=device)
+        p = DecodePlan(max_degree, torch.zeros(batch, **i32), torch.full((batch, max_degree), -1, **i32),
+                       torch.zeros(batch, **i32), torch.zeros(1, **i32))
+        p.c = _DecodePlanC(max_degree, p.count.data_ptr(), p.page.data_ptr(), p.block.data_ptr(), p.status.data_ptr())
+        return p
+
+
+def plan_decode(seqlens: torch.Tensor, page_table: torch.Tensor, cfg: Optional[RouteCfg] = None,
+                plan: Optional[DecodePlan] = None, stream=None) -> DecodePlan:
+    """bf1_plan_decode: page list of the newest token's block for every sequence."""
+    cfg = cfg or RouteCfg()
+    assert seqlens.is_cuda and seqlens.dtype == torch.int32 and page_table.dtype == torch.int32
+    batch, max_pages = page_table.shape
+    if plan is None:
+        _, deg = route_capacity(1, max_pages * 64, max_pages * 64, cfg)
+        plan = DecodePlan.empty(batch, deg, seqlens.device)
+    _check(load().bf1_plan_decode(seqlens.data_ptr(), page_table.data_ptr(), max_pages, batch, ctypes.byref(cfg),
+                                  ctypes.byref(plan.c), _stream_ptr(stream)))
+    return plan
+
+
+def decode_workspace(batch: int, hkv: int, max_degree: int, d: int, device) -> torch.Tensor:
+    """Zero-initialised scratch for decode_fwd (reusable across calls that do not overlap)."""
+    nbytes = int(load().bf1_decode_workspace_bytes(batch, hkv, max_degree, d))
+    return torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
+
+
+def decode_fwd(q, k_pages, v_pages, seqlens, plan: DecodePlan, workspace, scale: Optional[float] = None,
+               out=None, lse=None, stream=None):
+    """bf1_decode_fwd.  q [batch, hq, d]; k_pages / v_pages [pages, 64, hkv, d] bf16 CUDA."""
+    batch, hq, d = q.shape
+    num_pages, page, hkv, d2 = k_pages.shape
+    assert page == 64 and d2 == d and v_pages.shape == k_pages.shape
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((hq, batch), dtype=torch.float32, device=q.device)
+    _check(load().bf1_decode_fwd(q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), num_pages, seqlens.data_ptr(),
+                                 batch, hq, hkv, d, float(scale) if scale else 0.0, ctypes.byref(plan.c),
+                                 workspace.data_ptr(), out.data_ptr(), lse.data_ptr(), _stream_ptr(stream)))
     return out, lse
 
 

@@ -1,0 +1,280 @@
+// BF1 cached one-token decode over selected KV pages (paper Section 3.2 and 5.4).
+//
+// The newest token of a sequence of n cached tokens (position n-1, block j = (n-1) / 64) reads
+// the pages of P(j) -- O(log B) pages, O(b d log B) key/value elements per head -- out of a paged
+// KV cache: page = 64 tokens, [page, 64, Hkv, d] bf16, logical block -> physical page through a
+// page table.  The page list only changes when n crosses a block boundary, so the plan
+// (bf1_plan_decode) is made once per 64-token "route epoch" and reused by every decode step in
+// it; the attention call reads the current lengths itself to find how many tokens of the self
+// page are valid.  The paper measures planning at 100-121 us against 12-23 us of execution and
+// names plan reuse across the epoch as the open problem; here the plan is a 2-3 us kernel and is
+// off the per-token path.
+//
+// The work is memory-bound (every selected K/V byte is read once, 2*G MACs per element), so
+// there are no tensor cores here: one CTA per (sequence, KV head, list entry) streams one K page
+// and one V page through shared memory, computes the two grouped query heads' scores and a
+// partial (max, sum, O) triple; the last CTA of a (sequence, KV head) to finish combines the
+// partials (split-KV, combine by atomic ticket) and writes O and LSE.
+#include "bf1_common.cuh"
+
+namespace bf1 {
+
+constexpr int kPage = 64;             // tokens per page = block width b
+constexpr int kDecThreads = 128;
+
+struct DecodeArgs {
+    const __nv_bfloat16* q;           // [batch, hq, d]
+    const __nv_bfloat16* k_pages;     // [pages, 64, hkv, d]
+    const __nv_bfloat16* v_pages;
+    const int32_t* seqlens;           // [batch] current cached lengths (>= 0)
+    const int32_t* count;             // plan: [batch] pages to read
+    const int32_t* page;              // plan: [batch, max_degree] physical pages, self page last
+    const int32_t* block;             // plan: [batch] block index the plan was made for
+    int32_t* status;
+    int32_t max_degree, hq, hkv, num_pages;
+    float scale_log2;
+    float* part;                      // [batch, hkv, max_degree, 2, d + 2] partial (o[d], m, l)
+    int32_t* ticket;                  // [batch, hkv], zero before and after every call
+    __nv_bfloat16* o;                 // [batch, hq, d]
+    float* lse;                       // [hq, batch]
+    int32_t batch;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a) {
+    constexpr int kRowWords = D / 2;                    // 32-bit words per K/V row
+    __shared__ uint32_t sK[kPage][kRowWords + 1];       // +1 word: rows start in different banks
+    __shared__ uint32_t sV[kPage][kRowWords];
+    __shared__ float sQ[2][D];
+    __shared__ float sP[2][kPage];
+    __shared__ float sRed[2][2];
+    __shared__ int sLast;
+
+    const int e = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    const int tid = threadIdx.x;
+    const int cnt = a.count[s];
+    if (e >= cnt) return;
+    const int n = a.seqlens[s];
+    const int j = (n - 1) / kPage;
+    if (j != a.block[s]) {            // the plan belongs to another route epoch
+        if (tid == 0 && e == 0 && kvh == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+        return;
+    }
+    int pg = a.page[(size_t)s * a.max_degree + e];
+    if (pg < 0 || pg >= a.num_pages) {
+        if (tid == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+        pg = 0;
+    }
+    const int valid = (e == cnt - 1) ? (n - j * kPage) : kPage;   // self page: tokens up to n-1 only
+
+    // ---- stage q (2 heads), the K page and the V page of this KV head --------------------
+    for (int i = tid; i < 2 * D; i += kDecThreads)
+        sQ[i / D][i % D] = __bfloat162float(a.q[((size_t)s * a.hq + kvh * 2 + i / D) * D + i % D]);
+    {
+        constexpr int kVecPerRow = D / 8;               // 16-byte vectors per row
+        const size_t row_stride = (size_t)a.hkv * D;    // elements between consecutive tokens of a page
+        const __nv_bfloat16* kp = a.k_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
+        const __nv_bfloat16* vp = a.v_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
+        for (int i = tid; i < kPage * kVecPerRow; i += kDecThreads) {
+            const int r = i / kVecPerRow, c = i % kVecPerRow;
+            const uint4 kv = *reinterpret_cast<const uint4*>(kp + r * row_stride + c * 8);
+            const uint4 vv = *reinterpret_cast<const uint4*>(vp + r * row_stride + c * 8);
+            sK[r][c * 4 + 0] = kv.x; sK[r][c * 4 + 1] = kv.y; sK[r][c * 4 + 2] = kv.z; sK[r][c * 4 + 3] = kv.w;
+            *reinterpret_cast<uint4*>(&sV[r][c * 4]) = vv;
+        }
+    }
+    __syncthreads();
+
+    // ---- scores: thread = (head h, key r) ----------------------------------------------------
+    const int h = tid >> 6, r = tid & 63;
+    float sc = 0.f;
+#pragma unroll 8
+    for (int w = 0; w < kRowWords; ++w) {
+        const float2 kk = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&sK[r][w]));
+        sc = fmaf(sQ[h][2 * w], kk.x, sc);
+        sc = fmaf(sQ[h][2 * w + 1], kk.y, sc);
+    }
+    sc = (r < valid) ? sc * a.scale_log2 : -INFINITY;    // log2 domain
+    float mx = sc;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = mx;
+    __syncthreads();
+    mx = fmaxf(sRed[h][0], sRed[h][1]);                  // finite: key 0 of every page is valid
+    const float p = exp2f(sc - mx);
+    sP[h][r] = p;
+    float sum = p;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    __syncthreads();                                     // sRed reads done, sP written
+    if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = sum;
+    __syncthreads();
+    sum = sRed[h][0] + sRed[h][1];
+
+    // ---- partial O: thread = (head h, D / 64 output columns starting at c0) -------------------
+    constexpr int kColsPerThread = D / 64;
+    const int c0 = r * kColsPerThread;
+    float acc[kColsPerThread];
+#pragma unroll
+    for (int c = 0; c < kColsPerThread; ++c) acc[c] = 0.f;
+    const __nv_bfloat16* sVh = reinterpret_cast<const __nv_bfloat16*>(&sV[0][0]);
+    for (int k = 0; k < valid; ++k) {
+        const float pk = sP[h][k];
+#pragma unroll
+        for (int c = 0; c < kColsPerThread; ++c) acc[c] = fmaf(pk, __bfloat162float(sVh[k * D + c0 + c]), acc[c]);
+    }
+    float* my = a.part + ((((size_t)s * a.hkv + kvh) * a.max_degree + e) * 2 + h) * (D + 2);
+#pragma unroll
+    for (int c = 0; c < kColsPerThread; ++c) my[c0 + c] = acc[c];
+    if (r == 0) { my[D] = mx; my[D + 1] = sum; }
+
+    // ---- the last CTA of this (sequence, KV head) combines --------------------------------------
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int t = atomicAdd(a.ticket + s * a.hkv + kvh, 1);
+        sLast = (t == cnt - 1);
+        if (sLast) a.ticket[s * a.hkv + kvh] = 0;        // ready for the next call
+    }
+    __syncthreads();
+    if (!sLast) return;
+    __threadfence();
+    const float* base = a.part + (((size_t)s * a.hkv + kvh) * a.max_degree * 2 + h) * (D + 2);
+    const size_t estride = 2 * (D + 2);
+    float m_all = -INFINITY;
+    for (int i = 0; i < cnt; ++i) m_all = fmaxf(m_all, base[i * estride + D]);
+    float l_all = 0.f;
+    float out[kColsPerThread];
+#pragma unroll
+    for (int c = 0; c < kColsPerThread; ++c) out[c] = 0.f;
+    for (int i = 0; i < cnt; ++i) {                      // ascending list order: a fixed, data-independent order
+        const float w = exp2f(base[i * estride + D] - m_all);
+        l_all = fmaf(w, base[i * estride + D + 1], l_all);
+#pragma unroll
+        for (int c = 0; c < kColsPerThread; ++c) out[c] = fmaf(w, base[i * estride + c0 + c], out[c]);
+    }
+    const float inv = 1.f / l_all;
+    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + kvh * 2 + h) * D;
+#pragma unroll
+    for (int c = 0; c < kColsPerThread; ++c) orow[c0 + c] = __float2bfloat16_rn(out[c] * inv);
+    if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+}
+
+// One thread per sequence: Eq. 1 for the block of the newest token, mapped through the page table.
+__global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_table, int max_pages_per_seq,
+                                   int batch, bf1_route_cfg cfg, bf1_decode_plan plan) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s == 0) *plan.status = 0;
+    if (s >= batch) return;
+    const int n = seqlens[s];
+    int32_t* list = plan.page + (size_t)s * plan.max_degree;
+    int deg = 0;
+    int bad = 0;
+    const int j = n > 0 ? (n - 1) / kPage : -1;
+    if (n < 0 || j >= max_pages_per_seq) bad = BF1_DEV_BAD_SEQLENS;
+    if (n > 0 && !bad) {
+        int last = -1, kmax = -1;
+        if (cfg.dyadic) while ((1 << (kmax + 1)) <= j) ++kmax;
+        int g = cfg.global_first ? 0 : 0x7fffffff;
+        int k = kmax;
+        int l = max(j - cfg.local_blocks, 0);
+        while (true) {                                   // merge of the three ascending candidate streams
+            const int dcur = (k >= 0) ? j - (1 << k) : 0x7fffffff;
+            const int lcur = (l <= j) ? l : 0x7fffffff;
+            const int m = min(g, min(dcur, lcur));
+            if (m == 0x7fffffff) break;
+            if (m == g) g = 0x7fffffff;
+            if (m == dcur) --k;
+            if (m == lcur) ++l;
+            if (m != last) {
+                if (deg < plan.max_degree) list[deg] = page_table[(size_t)s * max_pages_per_seq + m];
+                else bad |= BF1_DEV_CAPACITY;
+                ++deg;
+                last = m;
+            }
+        }
+        if (deg > plan.max_degree) deg = plan.max_degree;
+    }
+    for (int e2 = deg; e2 < plan.max_degree; ++e2) list[e2] = -1;
+    plan.count[s] = bad ? 0 : deg;
+    plan.block[s] = j;
+    if (bad) atomicOr(plan.status, bad);
+}
+
+int check_cfg(const bf1_route_cfg* cfg);   // bf1_plan.cu
+
+}  // namespace bf1
+
+using namespace bf1;
+
+extern "C" int64_t bf1_decode_workspace_bytes(int32_t batch, int32_t hkv, int32_t max_degree, int32_t d) {
+    if (batch < 0 || hkv <= 0 || max_degree <= 0 || d <= 0) return -1;
+    const int64_t part = (int64_t)batch * hkv * max_degree * 2 * (d + 2) * (int64_t)sizeof(float);
+    const int64_t tick = (int64_t)batch * hkv * (int64_t)sizeof(int32_t);
+    return ((part + 255) / 256) * 256 + tick;
+}
+
+extern "C" int bf1_plan_decode(const int32_t* seqlens_dev, const int32_t* page_table_dev, int32_t max_pages_per_seq,
+                               int32_t batch, const bf1_route_cfg* cfg, const bf1_decode_plan* out, void* stream) {
+    if (int rc = check_cfg(cfg)) return rc;
+    if (!seqlens_dev || !page_table_dev || !out || !out->count || !out->page || !out->block || !out->status)
+        return fail(BF1_ERR_INVALID_ARG, "a decode-plan pointer is null");
+    if (batch < 0 || max_pages_per_seq < 1 || out->max_degree < 1)
+        return fail(BF1_ERR_INVALID_ARG, "bad batch, max_pages_per_seq or max_degree");
+    int32_t cap = 0, need = 0;
+    if (int rc = bf1_route_capacity(1, (int64_t)max_pages_per_seq * kPage, max_pages_per_seq * kPage, cfg, &cap, &need))
+        return rc;
+    if (out->max_degree < need)
+        return fail(BF1_ERR_CAPACITY, "decode plan max_degree %d < %d needed for %d pages per sequence", out->max_degree,
+                    need, max_pages_per_seq);
+    if (batch == 0) return BF1_OK;
+    plan_decode_kernel<<<(batch + 127) / 128, 128, 0, (cudaStream_t)stream>>>(seqlens_dev, page_table_dev,
+                                                                               max_pages_per_seq, batch, *cfg, *out);
+    BF1_CUDA_CHECK(cudaGetLastError());
+    return BF1_OK;
+}
+
+extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_pages, int32_t num_pages,
+                              const int32_t* seqlens_dev, int32_t batch, int32_t hq, int32_t hkv, int32_t d,
+                              float softmax_scale, const bf1_decode_plan* plan, void* workspace, void* o, float* lse,
+                              void* stream) {
+    if (!q || !k_pages || !v_pages || !seqlens_dev || !plan || !workspace || !o || !lse)
+        return fail(BF1_ERR_INVALID_ARG, "a pointer is null");
+    if (!plan->count || !plan->page || !plan->block || !plan->status)
+        return fail(BF1_ERR_INVALID_ARG, "a decode-plan pointer is null");
+    if (batch < 0 || num_pages < 0 || hq <= 0 || hkv <= 0) return fail(BF1_ERR_INVALID_ARG, "negative or zero size argument");
+    if (hq % hkv != 0) return fail(BF1_ERR_INVALID_ARG, "hq %d is not a multiple of hkv %d", hq, hkv);
+    if (hq / hkv != 2) return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 is supported", hq / hkv);
+    if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
+    if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)o | (uintptr_t)workspace) & 15)
+        return fail(BF1_ERR_INVALID_ARG, "q, k_pages, v_pages, o and workspace must be 16-byte aligned");
+    if (plan->max_degree < 1 || plan->max_degree > 65535 || hkv > 65535 || batch > 65535)
+        return fail(BF1_ERR_UNSUPPORTED, "max_degree, hkv and batch must fit the grid (<= 65535)");
+    if (batch == 0) return BF1_OK;
+    DecodeArgs a;
+    a.q = (const __nv_bfloat16*)q;
+    a.k_pages = (const __nv_bfloat16*)k_pages;
+    a.v_pages = (const __nv_bfloat16*)v_pages;
+    a.seqlens = seqlens_dev;
+    a.count = plan->count;
+    a.page = plan->page;
+    a.block = plan->block;
+    a.status = plan->status;
+    a.max_degree = plan->max_degree;
+    a.hq = hq;
+    a.hkv = hkv;
+    a.num_pages = num_pages;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.part = (float*)workspace;
+    const int64_t part = (int64_t)batch * hkv * plan->max_degree * 2 * (d + 2) * (int64_t)sizeof(float);
+    a.ticket = (int32_t*)((char*)workspace + ((part + 255) / 256) * 256);
+    a.o = (__nv_bfloat16*)o;
+    a.lse = lse;
+    a.batch = batch;
+    dim3 grid(plan->max_degree, hkv, batch);
+    if (d == 128) decode_kernel<128><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
+    else decode_kernel<64><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
+    BF1_CUDA_CHECK(cudaGetLastError());
+    return BF1_OK;
+}
