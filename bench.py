@@ -226,6 +226,65 @@ def sweep(bf1, dev):
     return out
 
 
+def decode_sweep(bf1, dev):
+    """Selected-page one-token decode (Section 5.4, Table 3's grid: 32K / 64K context, batch 1 / 8 / 32).
+    A pool of 8192 physical pages (2.1 GB of K and V, far larger than L2) and 32 random page tables per
+    point; the 32 decode calls (each with its own plan, so each reads different, mostly cold pages) are
+    captured in one CUDA graph so that host launch latency does not hide the kernel, and the graph's
+    time is divided by 32.  Planning is timed the same way, on its own: one plan serves a whole
+    64-token route epoch.  Bytes = selected K and V pages, read once."""
+    out = []
+    hq, hkv, d, reps = 16, 8, 128, 32
+    peaks = measured_peaks()
+    g = torch.Generator(device=dev)
+    g.manual_seed(777)
+    pool = 8192
+    k_pages = torch.randn((pool, 64, hkv, d), generator=g, device=dev, dtype=torch.bfloat16)
+    v_pages = torch.randn((pool, 64, hkv, d), generator=g, device=dev, dtype=torch.bfloat16)
+    side = torch.cuda.Stream(device=dev)
+    for n in (32768, 65536):
+        for batch in (1, 8, 32):
+            nb = n // 64
+            q = torch.randn((batch, hq, d), generator=g, device=dev, dtype=torch.bfloat16)
+            sl = torch.full((batch,), n, dtype=torch.int32, device=dev)
+            tables = [torch.randint(0, pool, (batch, nb), generator=g, device=dev, dtype=torch.int32) for _ in range(reps)]
+            plans = [bf1.plan_decode(sl, t) for t in tables]
+            ws = bf1.decode_workspace(batch, hkv, plans[0].max_degree, d, dev)
+            o = torch.empty_like(q)
+            lse = torch.empty((hq, batch), dtype=torch.float32, device=dev)
+            torch.cuda.synchronize()
+            timings = {}
+            for what in ("plan", "decode"):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    calls = (lambda i: bf1.plan_decode(sl, tables[i], plan=plans[i])) if what == "plan" else \
+                            (lambda i: bf1.decode_fwd(q, k_pages, v_pages, sl, plans[i], ws, out=o, lse=lse))
+                    for i in range(2):
+                        calls(i)
+                    side.synchronize()
+                    with torch.cuda.graph(graph, stream=side):
+                        for i in range(reps):
+                            calls(i)
+                    ts = []
+                    for _ in range(8):
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record(side)
+                        graph.replay()
+                        e1.record(side)
+                        e1.synchronize()
+                        ts.append(e0.elapsed_time(e1) / reps)
+                timings[what] = statistics.median(ts[2:])
+            assert all(int(p.status.item()) == 0 for p in plans)
+            nbytes = int(plans[0].count.sum().item()) * 64 * hkv * d * 2 * 2
+            ms = timings["decode"]
+            out.append({"context": n, "batch": batch, "pages_per_seq": int(plans[0].count[0].item()),
+                        "plan_us": round(timings["plan"] * 1e3, 2), "decode_us": round(ms * 1e3, 2),
+                        "selected_kv_bytes": nbytes, "gbs": round(nbytes / ms / 1e6, 1),
+                        "frac_of_hbm_peak": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4),
+                        "timing": "32 calls on 32 random page tables in one CUDA graph, pool 2.1 GB"})
+    return out
+
+
 def run_single(args):
     """A few plain launches of one mode on one named workload (what the ncu captures run)."""
     import paper_2608_20427_b200 as bf1
@@ -389,6 +448,7 @@ def run_ours(args):
     }
     if not args.no_sweep and world == 1:
         line["sweep"] = sweep(bf1, dev)
+        line["decode"] = decode_sweep(bf1, dev)
     if not args.no_cpu and world == 1:
         q, k, v = I.draw_qkv(w)
         val, dt, desc, thr = oracle_rate(w, q, k, v, target_s=15.0)
