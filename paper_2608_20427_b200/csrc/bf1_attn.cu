@@ -289,6 +289,35 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         tma_prefetch_desc(&tm_o);
     }
     __syncwarp();
+    // The scheduler warp decodes this CTA's first unit (unit blockIdx.x; the shared counter hands
+    // out the units after the first gridDim.x) while the others set up barriers and tensor memory:
+    // the decode is a chain of dependent global loads that would otherwise delay the first copy.
+    auto fetch_unit = [&](int u, int nqb_, Unit& un, int& my_p) {
+        decode_unit(args, nqb_, u, un);
+        my_p = 0;
+        if (lane < un.cnt) {   // entries 0..31, one per lane, made safe to use
+            int p = args.dense ? lane : un.list[lane];
+            if (p < 0 || p > un.j || (lane == un.cnt - 1) != (p == un.j)) {
+                if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
+                p = (lane == un.cnt - 1) ? un.j : 0;
+            }
+            my_p = p;
+        }
+    };
+    Unit un0 = {};
+    int my_p0 = 0;
+    bool have0 = false;
+    if (warp == 2) {
+        int nqb0 = 0;
+        if (!args.dense) {
+            nqb0 = min(*args.num_qblocks, args.capacity);
+        } else {
+            for (int s = 0; s < args.batch; ++s)
+                nqb0 += (args.cu_seqlens[s + 1] - args.cu_seqlens[s] + kBlock - 1) / kBlock;
+        }
+        have0 = (int)blockIdx.x < nqb0 * args.hkv;
+        if (have0) fetch_unit(blockIdx.x, nqb0, un0, my_p0);
+    }
     if (warp == 1) {
         tmem_alloc(smem_u32(s_tmem_base), C::kTmemCols);
         tmem_relinquish();
@@ -309,29 +338,25 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         if (warp == 2) {
             // ================================ scheduler =======================================
             for (int n = 0;; ++n) {
-                int u = 0;
-                if (lane == 0) u = args.sched ? atomicAdd(args.sched, 1) : (int)(blockIdx.x + n * gridDim.x);
-                u = __shfl_sync(0xffffffffu, u, 0);
-                const bool have = u < total_units && !*abort_flag;
-                Unit un = {};
-                int my_p = 0;
-                if (have) {
-                    decode_unit(args, nqb, u, un);
-                    if (lane < un.cnt) {   // entries 0..31, one per lane, made safe to use
-                        int p = args.dense ? lane : un.list[lane];
-                        if (p < 0 || p > un.j || (lane == un.cnt - 1) != (p == un.j)) {
-                            if (args.status) atomicOr(args.status, BF1_DEV_BAD_ROUTE);
-                            p = (lane == un.cnt - 1) ? un.j : 0;
-                        }
-                        my_p = p;
-                        if (kPrefetchMode >= 2) {
-                            // pull this block into L2 ahead of the real load (needs no shared memory)
-                            const int row = un.seq0 + p * kBlock;
-                            tma_prefetch_l2_4d(&tm_k, 0, row, un.kvh, 0);
-                            tma_prefetch_l2_4d(&tm_v, 0, row, un.kvh, 0);
-                        }
+                Unit un = un0;
+                int my_p = my_p0;
+                bool have = have0 && !*abort_flag;
+                if (n > 0) {
+                    int u = 0;
+                    if (lane == 0)
+                        u = (args.sched ? atomicAdd(args.sched, 1) + (int)gridDim.x : (int)(blockIdx.x + n * gridDim.x));
+                    u = __shfl_sync(0xffffffffu, u, 0);
+                    have = u < total_units && !*abort_flag;
+                    if (have) fetch_unit(u, nqb, un, my_p);
+                }
+                if (have && kPrefetchMode >= 1) {
+                    if (lane == 0) tma_prefetch_l2_4d(&tm_q, 0, un.tok0, un.kvh * 2, 0);
+                    if (kPrefetchMode >= 2 && lane < un.cnt) {
+                        // pull this block into L2 ahead of the real load (needs no shared memory)
+                        const int row = un.seq0 + my_p * kBlock;
+                        tma_prefetch_l2_4d(&tm_k, 0, row, un.kvh, 0);
+                        tma_prefetch_l2_4d(&tm_v, 0, row, un.kvh, 0);
                     }
-                    if (kPrefetchMode >= 1 && lane == 0) tma_prefetch_l2_4d(&tm_q, 0, un.tok0, un.kvh * 2, 0);
                 }
                 const int qs = n % kQueue;
                 if (n >= kQueue) mbar_wait(bar_sq_free + 8 * qs, ((n / kQueue) - 1) & 1, abort_flag, args.status);
