@@ -285,11 +285,43 @@ def decode_sweep(bf1, dev):
     return out
 
 
+def run_single_decode(args, bf1, dev):
+    """A few plain decode calls at batch 32, context 32768, each on its own random page table."""
+    hq, hkv, d, batch, n, pool = 16, 8, 128, 32, 32768, 8192
+    g = torch.Generator(device=dev)
+    g.manual_seed(778)
+    k_pages = torch.randn((pool, 64, hkv, d), generator=g, device=dev, dtype=torch.bfloat16)
+    v_pages = torch.randn((pool, 64, hkv, d), generator=g, device=dev, dtype=torch.bfloat16)
+    q = torch.randn((batch, hq, d), generator=g, device=dev, dtype=torch.bfloat16)
+    sl = torch.full((batch,), n, dtype=torch.int32, device=dev)
+    total = args.warmup + args.steps
+    tables = [torch.randint(0, pool, (batch, n // 64), generator=g, device=dev, dtype=torch.int32) for _ in range(total)]
+    plans = [bf1.plan_decode(sl, t) for t in tables]
+    ws = bf1.decode_workspace(batch, hkv, plans[0].max_degree, d, dev)
+    o = torch.empty_like(q)
+    lse = torch.empty((hq, batch), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    ts = []
+    for i in range(total):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        bf1.decode_fwd(q, k_pages, v_pages, sl, plans[i], ws, out=o, lse=lse)
+        e1.record(stream)
+        e1.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    nbytes = int(plans[0].count.sum().item()) * 64 * hkv * d * 2 * 2
+    ms = statistics.median(ts[args.warmup:])
+    print(json.dumps({"single": "decode batch 32 context 32768", "ms": ms, "steps": args.steps,
+                      "selected_kv_bytes": nbytes, "gbs_incl_launch_latency": nbytes / ms / 1e6}))
+
+
 def run_single(args):
     """A few plain launches of one mode on one named workload (what the ncu captures run)."""
     import paper_2608_20427_b200 as bf1
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
+    if args.mode == "decode":
+        return run_single_decode(args, bf1, dev)
     w = I.WORKLOADS[args.single]
     q, k, v = (t.to(dev) for t in I.draw_qkv(w))
     cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
@@ -469,7 +501,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--single", default=None, choices=sorted(I.WORKLOADS),
                     help="only time `--steps` launches of one workload (used for profiling)")
-    ap.add_argument("--mode", default="bf1", choices=["bf1", "dense"])
+    ap.add_argument("--mode", default="bf1", choices=["bf1", "dense", "decode"])
     args = ap.parse_args()
     if args.single:
         run_single(args)

@@ -7,7 +7,7 @@
 // (bf1_plan_decode) is made once per 64-token "route epoch" and reused by every decode step in
 // it; the attention call reads the current lengths itself to find how many tokens of the self
 // page are valid.  The paper measures planning at 100-121 us against 12-23 us of execution and
-// names plan reuse across the epoch as the open problem; here the plan is a 2-3 us kernel and is
+// names plan reuse across the epoch as the open problem; here the plan is a ~4 us kernel and is
 // off the per-token path.
 //
 // The work is memory-bound (every selected K/V byte is read once, 2*G MACs per element), so
@@ -43,58 +43,79 @@ struct DecodeArgs {
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a) {
     constexpr int kRowWords = D / 2;                    // 32-bit words per K/V row
-    __shared__ uint32_t sK[kPage][kRowWords + 1];       // +1 word: rows start in different banks
-    __shared__ uint32_t sV[kPage][kRowWords];
-    __shared__ float sQ[2][D];
-    __shared__ float sP[2][kPage];
+    constexpr int kVecPerRow = D / 8;                   // 16-byte vectors per row
+    constexpr int kVecPerThread = kPage * kVecPerRow / kDecThreads;
+    // K rows are read whole by one thread each (16 bytes at a time), so their 16-byte chunks are
+    // XOR-swizzled with the row index to keep 8 neighbouring rows in different banks
+    __shared__ __align__(16) uint32_t sK[kPage][kRowWords];
+    __shared__ __align__(16) uint32_t sV[kPage][kRowWords];
+    __shared__ __align__(16) float sQ[2][D];
+    __shared__ __align__(16) float sP[2][kPage];
     __shared__ float sRed[2][2];
+    __shared__ float sW[2][64];                         // combine: weight of every partial
     __shared__ int sLast;
 
     const int e = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x;
+    // the four scalars this CTA needs are independent loads: issue them together
     const int cnt = a.count[s];
-    if (e >= cnt) return;
     const int n = a.seqlens[s];
+    const int planned = a.block[s];
+    int pg = a.page[(size_t)s * a.max_degree + e];
+    if (e >= cnt) return;
     const int j = (n - 1) / kPage;
-    if (j != a.block[s]) {            // the plan belongs to another route epoch
+    if (j != planned) {               // the plan belongs to another route epoch
         if (tid == 0 && e == 0 && kvh == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
         return;
     }
-    int pg = a.page[(size_t)s * a.max_degree + e];
     if (pg < 0 || pg >= a.num_pages) {
         if (tid == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
         pg = 0;
     }
     const int valid = (e == cnt - 1) ? (n - j * kPage) : kPage;   // self page: tokens up to n-1 only
 
-    // ---- stage q (2 heads), the K page and the V page of this KV head --------------------
-    for (int i = tid; i < 2 * D; i += kDecThreads)
-        sQ[i / D][i % D] = __bfloat162float(a.q[((size_t)s * a.hq + kvh * 2 + i / D) * D + i % D]);
+    // ---- stage q (2 heads), the K page and the V page of this KV head: every load of the thread
+    //      is in flight before the first one is used ---------------------------------------------
     {
-        constexpr int kVecPerRow = D / 8;               // 16-byte vectors per row
         const size_t row_stride = (size_t)a.hkv * D;    // elements between consecutive tokens of a page
         const __nv_bfloat16* kp = a.k_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
         const __nv_bfloat16* vp = a.v_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
-        for (int i = tid; i < kPage * kVecPerRow; i += kDecThreads) {
-            const int r = i / kVecPerRow, c = i % kVecPerRow;
-            const uint4 kv = *reinterpret_cast<const uint4*>(kp + r * row_stride + c * 8);
-            const uint4 vv = *reinterpret_cast<const uint4*>(vp + r * row_stride + c * 8);
-            sK[r][c * 4 + 0] = kv.x; sK[r][c * 4 + 1] = kv.y; sK[r][c * 4 + 2] = kv.z; sK[r][c * 4 + 3] = kv.w;
-            *reinterpret_cast<uint4*>(&sV[r][c * 4]) = vv;
+        uint4 kreg[kVecPerThread], vreg[kVecPerThread];
+#pragma unroll
+        for (int it = 0; it < kVecPerThread; ++it) {
+            const int i = tid + it * kDecThreads, r = i / kVecPerRow, c = i % kVecPerRow;
+            kreg[it] = *reinterpret_cast<const uint4*>(kp + r * row_stride + c * 8);
+            vreg[it] = *reinterpret_cast<const uint4*>(vp + r * row_stride + c * 8);
+        }
+        for (int i = tid; i < 2 * D; i += kDecThreads)
+            sQ[i / D][i % D] = __bfloat162float(a.q[((size_t)s * a.hq + kvh * 2 + i / D) * D + i % D]);
+#pragma unroll
+        for (int it = 0; it < kVecPerThread; ++it) {
+            const int i = tid + it * kDecThreads, r = i / kVecPerRow, c = i % kVecPerRow;
+            *reinterpret_cast<uint4*>(&sK[r][(c ^ (r & 7)) * 4]) = kreg[it];
+            *reinterpret_cast<uint4*>(&sV[r][c * 4]) = vreg[it];
         }
     }
     __syncthreads();
 
     // ---- scores: thread = (head h, key r) ----------------------------------------------------
     const int h = tid >> 6, r = tid & 63;
-    float sc = 0.f;
-#pragma unroll 8
-    for (int w = 0; w < kRowWords; ++w) {
-        const float2 kk = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&sK[r][w]));
-        sc = fmaf(sQ[h][2 * w], kk.x, sc);
-        sc = fmaf(sQ[h][2 * w + 1], kk.y, sc);
+    float sc0 = 0.f, sc1 = 0.f;
+#pragma unroll
+    for (int c = 0; c < kVecPerRow; ++c) {               // 8 elements per step: one 16-byte K load, two of q
+        const uint4 kw = *reinterpret_cast<const uint4*>(&sK[r][(c ^ (r & 7)) * 4]);
+        const float4 qa = *reinterpret_cast<const float4*>(&sQ[h][c * 8]);
+        const float4 qb = *reinterpret_cast<const float4*>(&sQ[h][c * 8 + 4]);
+        sc0 = fmaf(qa.x, __uint_as_float(kw.x << 16), sc0);                  // low half = even element
+        sc1 = fmaf(qa.y, __uint_as_float(kw.x & 0xffff0000u), sc1);
+        sc0 = fmaf(qa.z, __uint_as_float(kw.y << 16), sc0);
+        sc1 = fmaf(qa.w, __uint_as_float(kw.y & 0xffff0000u), sc1);
+        sc0 = fmaf(qb.x, __uint_as_float(kw.z << 16), sc0);
+        sc1 = fmaf(qb.y, __uint_as_float(kw.z & 0xffff0000u), sc1);
+        sc0 = fmaf(qb.z, __uint_as_float(kw.w << 16), sc0);
+        sc1 = fmaf(qb.w, __uint_as_float(kw.w & 0xffff0000u), sc1);
     }
-    sc = (r < valid) ? sc * a.scale_log2 : -INFINITY;    // log2 domain
+    const float sc = (r < valid) ? (sc0 + sc1) * a.scale_log2 : -INFINITY;   // log2 domain
     float mx = sc;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
@@ -111,17 +132,27 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
     __syncthreads();
     sum = sRed[h][0] + sRed[h][1];
 
-    // ---- partial O: thread = (head h, D / 64 output columns starting at c0) -------------------
-    constexpr int kColsPerThread = D / 64;
+    // ---- partial O: thread = (head h, D / 64 adjacent output columns) ---------------------------
+    constexpr int kColsPerThread = D / 64;               // 2 at d = 128 (one 32-bit word of V), 1 at d = 64
     const int c0 = r * kColsPerThread;
-    float acc[kColsPerThread];
+    float acc[2] = {0.f, 0.f};
+    if (kColsPerThread == 2) {
+        for (int k4 = 0; k4 < valid; k4 += 4) {          // never touch V rows past the newest token
+            const float4 pk = *reinterpret_cast<const float4*>(&sP[h][k4]);   // masked keys: p = 0
+            const float pv[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c) acc[c] = 0.f;
-    const __nv_bfloat16* sVh = reinterpret_cast<const __nv_bfloat16*>(&sV[0][0]);
-    for (int k = 0; k < valid; ++k) {
-        const float pk = sP[h][k];
-#pragma unroll
-        for (int c = 0; c < kColsPerThread; ++c) acc[c] = fmaf(pk, __bfloat162float(sVh[k * D + c0 + c]), acc[c]);
+            for (int q4 = 0; q4 < 4; ++q4) {
+                if (k4 + q4 < valid) {
+                    const uint32_t vw = sV[k4 + q4][r];
+                    acc[0] = fmaf(pv[q4], __uint_as_float(vw << 16), acc[0]);
+                    acc[1] = fmaf(pv[q4], __uint_as_float(vw & 0xffff0000u), acc[1]);
+                }
+            }
+        }
+    } else {
+        const __nv_bfloat16* sVh = reinterpret_cast<const __nv_bfloat16*>(&sV[0][0]);
+#pragma unroll 8
+        for (int k = 0; k < valid; ++k) acc[0] = fmaf(sP[h][k], __bfloat162float(sVh[k * D + c0]), acc[0]);
     }
     float* my = a.part + ((((size_t)s * a.hkv + kvh) * a.max_degree + e) * 2 + h) * (D + 2);
 #pragma unroll
@@ -141,15 +172,28 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
     __threadfence();
     const float* base = a.part + (((size_t)s * a.hkv + kvh) * a.max_degree * 2 + h) * (D + 2);
     const size_t estride = 2 * (D + 2);
+    // every partial's (max, sum) is fetched by its own thread, so the loads overlap
+    if (r < cnt) sW[h][r] = base[r * estride + D];
+    __syncthreads();
     float m_all = -INFINITY;
-    for (int i = 0; i < cnt; ++i) m_all = fmaxf(m_all, base[i * estride + D]);
-    float l_all = 0.f;
-    float out[kColsPerThread];
+    for (int i = 0; i < cnt && i < 64; ++i) m_all = fmaxf(m_all, sW[h][i]);
+    float wgt = 0.f, lpart = 0.f;
+    if (r < cnt) {
+        wgt = exp2f(sW[h][r] - m_all);
+        lpart = wgt * base[r * estride + D + 1];
+    }
+    __syncthreads();
+    if (r < cnt) sW[h][r] = wgt;
+    float l_all = lpart;                                 // sum over the (at most 64) partials of this head
 #pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c) out[c] = 0.f;
-    for (int i = 0; i < cnt; ++i) {                      // ascending list order: a fixed, data-independent order
-        const float w = exp2f(base[i * estride + D] - m_all);
-        l_all = fmaf(w, base[i * estride + D + 1], l_all);
+    for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xffffffffu, l_all, off);
+    if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = l_all;
+    __syncthreads();
+    l_all = sRed[h][0] + sRed[h][1];
+    float out[2] = {0.f, 0.f};
+#pragma unroll 4
+    for (int i = 0; i < cnt; ++i) {                      // ascending list order: fixed and data-independent
+        const float w = sW[h][i];
 #pragma unroll
         for (int c = 0; c < kColsPerThread; ++c) out[c] = fmaf(w, base[i * estride + c0 + c], out[c]);
     }
@@ -248,8 +292,8 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
     if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)o | (uintptr_t)workspace) & 15)
         return fail(BF1_ERR_INVALID_ARG, "q, k_pages, v_pages, o and workspace must be 16-byte aligned");
-    if (plan->max_degree < 1 || plan->max_degree > 65535 || hkv > 65535 || batch > 65535)
-        return fail(BF1_ERR_UNSUPPORTED, "max_degree, hkv and batch must fit the grid (<= 65535)");
+    if (plan->max_degree < 1 || plan->max_degree > 64 || hkv > 65535 || batch > 65535)
+        return fail(BF1_ERR_UNSUPPORTED, "max_degree must be <= 64; hkv and batch must fit the grid (<= 65535)");
     if (batch == 0) return BF1_OK;
     DecodeArgs a;
     a.q = (const __nv_bfloat16*)q;

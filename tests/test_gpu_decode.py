@@ -112,6 +112,28 @@ def test_page_permutation_invariance_and_zero_decoy_leakage():
         assert np.array_equal(out, ref[0]) and np.array_equal(lse, ref[1])
 
 
+def test_unwritten_page_tails_may_hold_anything():
+    """The part of the newest page behind the newest token is unwritten cache memory: NaN there
+    (and in pages the route does not select) must not reach the output."""
+    w = I.custom([1000, 65], hq=4, hkv=2, d=128, seed=3400)
+    q, k, v = I.draw_qkv(w)
+    k_pages, v_pages, table = paged_cache(w, k, v, seed=4)
+    out0, lse0, _, _ = run_decode(w, q, k_pages, v_pages, table)
+    used = set(int(x) for x in table.flatten().tolist() if x >= 0)
+    for pg in range(k_pages.shape[0]):
+        if pg not in used:
+            k_pages[pg] = float("nan")
+            v_pages[pg] = float("nan")
+    for s, n in enumerate(w.seqlens):
+        tail = n % 64
+        if tail:
+            pg = int(table[s, (n - 1) // 64])
+            k_pages[pg, tail:] = float("nan")
+            v_pages[pg, tail:] = float("nan")
+    out1, lse1, _, _ = run_decode(w, q, k_pages, v_pages, table)
+    assert np.array_equal(out0, out1) and np.array_equal(lse0, lse1)
+
+
 def test_one_plan_serves_a_route_epoch_and_refuses_the_next():
     n0 = 64 * 9 + 1                                       # first token of block 9
     w = I.custom([n0 + 63], hq=4, hkv=2, d=128, seed=3300)
