@@ -69,6 +69,9 @@ def lib():
             f = getattr(L, "bf1o_attn_route" + suf)
             f.restype = None
             f.argtypes = [cp, vp, vp, vp, vp, i32, i32, i32, i32, f64, vp, i64, vp, vp]
+            f = getattr(L, "bf1o_attn_route_bwd" + suf)
+            f.restype = None
+            f.argtypes = [cp, vp, vp, vp, vp, vp, i32, i32, i32, i32, f64, vp, vp, vp]
             f = getattr(L, "bf1o_dense_causal" + suf)
             f.restype = None
             f.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, f64, vp, i64, vp, vp]
@@ -199,3 +202,21 @@ def dense_causal(q, k, v, cu_seqlens: Sequence[int], scale: Optional[float] = No
     f(_ptr(qb), _ptr(kb), _ptr(vb), _ptr(cu), len(cu) - 1, hq, hkv, d, _scale(scale, d),
       rp, nr, _ptr(o), _ptr(lse))
     return o, lse
+
+
+def attn_route_bwd(c: Cfg, q, k, v, d_o: np.ndarray, cu_seqlens: Sequence[int], scale: Optional[float] = None,
+                   fp64: bool = True):
+    """Gradients (dq, dk, dv) of the routed attention for an upstream gradient d_o [T, hq, d]."""
+    T, hq, d = q.shape
+    hkv = k.shape[1]
+    dtype = np.float64 if fp64 else np.float32
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    qb, kb, vb = bf16_bits(q), bf16_bits(k), bf16_bits(v)
+    go = np.ascontiguousarray(d_o.astype(dtype))
+    dq = np.empty((T, hq, d), dtype=dtype)
+    dk = np.empty((T, hkv, d), dtype=dtype)
+    dv = np.empty((T, hkv, d), dtype=dtype)
+    f = lib().bf1o_attn_route_bwd_f64 if fp64 else lib().bf1o_attn_route_bwd_f32
+    f(ctypes.byref(c), _ptr(qb), _ptr(kb), _ptr(vb), _ptr(go), _ptr(cu), len(cu) - 1, hq, hkv, d,
+      _scale(scale, d), _ptr(dq), _ptr(dk), _ptr(dv))
+    return dq, dk, dv
