@@ -209,6 +209,21 @@ int bf1_decode_fwd(const void *q, const void *k_pages, const void *v_pages, int3
                    float softmax_scale, const bf1_decode_plan *plan /* host */, void *workspace,
                    void *o, float *lse, void *stream);
 
+/* ---- backward over the same route (Section 4.2 gates on "forward and backward with finite Q/K/V
+ * gradients") -------------------------------------------------------------------------------------
+ * Given the forward's inputs, its outputs o and lse, and the upstream gradient d_o [T, hq, d] bf16,
+ * writes dq [T, hq, d], dk and dv [T, hkv, d] in bf16 (the gradients of the G query heads of a KV
+ * head add up in dk, dv).  P is recomputed as exp(scale * <q, k> - lse); dk and dv are accumulated
+ * in fp32 in `workspace` (bf1_attn_bwd_workspace_bytes() bytes, 16-byte aligned; it is cleared by
+ * the call) with floating-point atomics, so their last bits depend on the order of arrival.
+ * Head dimension 128 only; other limits as bf1_attn_fwd.  `route` must be the forward's. */
+int64_t bf1_attn_bwd_workspace_bytes(int64_t total_tokens, int32_t hkv, int32_t d);
+int bf1_attn_bwd(const void *q, const void *k, const void *v, const void *o, const float *lse,
+                 const void *d_o, const int32_t *cu_seqlens_dev, int32_t batch, int64_t total_tokens,
+                 int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d, float softmax_scale,
+                 const bf1_route *route /* host */, void *workspace, void *dq, void *dk, void *dv,
+                 void *stream);
+
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char *bf1_last_error(void);
 

@@ -20,7 +20,7 @@ DEV_BAD_SEQLENS, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_ROUTE = 1, 2, 4, 8
 
 EXPORTS = ("bf1_route_capacity", "bf1_plan_route", "bf1_attn_fwd", "bf1_dense_causal_fwd",
            "bf1_attn_fwd_noalloc", "bf1_plan_decode", "bf1_decode_workspace_bytes", "bf1_decode_fwd",
-           "bf1_last_error", "bf1_version")
+           "bf1_attn_bwd", "bf1_attn_bwd_workspace_bytes", "bf1_last_error", "bf1_version")
 
 
 class RouteCfg(ctypes.Structure):
@@ -83,6 +83,11 @@ def load():
     L.bf1_decode_fwd.restype = ctypes.c_int
     L.bf1_decode_fwd.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, f32, ctypes.POINTER(_DecodePlanC), vp, vp,
                                  vp, vp]
+    L.bf1_attn_bwd_workspace_bytes.restype = i64
+    L.bf1_attn_bwd_workspace_bytes.argtypes = [i64, i32, i32]
+    L.bf1_attn_bwd.restype = ctypes.c_int
+    L.bf1_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(_RouteC),
+                               vp, vp, vp, vp, vp]
     L.bf1_last_error.restype = ctypes.c_char_p
     L.bf1_last_error.argtypes = []
     L.bf1_version.restype = ctypes.c_int
@@ -280,6 +285,22 @@ def decode_fwd(q, k_pages, v_pages, seqlens, plan: DecodePlan, workspace, scale:
                                  batch, hq, hkv, d, float(scale) if scale else 0.0, ctypes.byref(plan.c),
                                  workspace.data_ptr(), out.data_ptr(), lse.data_ptr(), _stream_ptr(stream)))
     return out, lse
+
+
+def attn_bwd(q, k, v, o, lse, d_o, cu_seqlens, max_seqlen: int, route: Route, scale: Optional[float] = None,
+             workspace=None, stream=None):
+    """bf1_attn_bwd: (dq, dk, dv) in bf16 for the upstream gradient d_o; d = 128 only."""
+    T, hq, hkv, d = _check_qkv(q, k, v)
+    assert d_o.shape == q.shape and d_o.dtype == torch.bfloat16 and d_o.is_contiguous()
+    if workspace is None:
+        workspace = torch.empty(max(int(load().bf1_attn_bwd_workspace_bytes(T, hkv, d)), 16), dtype=torch.uint8,
+                                device=q.device)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    _check(load().bf1_attn_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
+                               cu_seqlens.data_ptr(), cu_seqlens.numel() - 1, T, max_seqlen, hq, hkv, d,
+                               float(scale) if scale else 0.0, ctypes.byref(route.c), workspace.data_ptr(),
+                               dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), _stream_ptr(stream)))
+    return dq, dk, dv
 
 
 def cu_seqlens_tensor(seqlens: Sequence[int], device) -> torch.Tensor:

@@ -816,6 +816,11 @@ static int make_store_map(CUtensorMap* m, void* ptr, int64_t T, int H, int d) {
     return BF1_OK;
 }
 
+// the same map for the other translation units of the library
+int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box) {
+    return make_map(m, ptr, T, H, d, heads_per_box);
+}
+
 struct DeviceInfo {
     int sm_count = 0;
     bool ok = false;

@@ -1,0 +1,364 @@
+// BF1 attention backward (dQ, dK, dV) over the same route, for sm_100a, head dimension 128.
+//
+// The paper gates its operator on "forward and backward with finite Q/K/V gradients" (Section
+// 4.2).  With P = exp(S - LSE) recomputed from the saved LSE and D_i = <dO_i, O_i>:
+//     dV_p += P^T dO,   dP = dO V_p^T,   dS = P o (dP - D) * scale,   dQ += dS K_p,   dK_p += dS^T Q.
+// Work unit = (query block, KV head) as in the forward pass: the two grouped query heads are the
+// 128 rows of every MMA, so their contributions to dK / dV add up inside the tensor core.  Per
+// list entry p, five groups of tcgen05 MMAs:
+//     S    = Q   K_p^T        (128 x 64 x 128)   A, B K-major from shared memory
+//     dP   = dO  V_p^T        (128 x 64 x 128)   same layouts
+//     dQ  += dS  K_p          (128 x 128 x 64)   A = dS (bf16, written to shared memory by the threads,
+//                                                K-major), B = K_p MN-major; accumulates in TMEM
+//     dV^T = dO^T P           (128 x 64 x 128)   A = dO MN-major, B = P MN-major (row-major [q][kv] tile)
+//     dK^T = Q^T  dS          (128 x 64 x 128)   A = Q MN-major,  B = dS MN-major
+// dV^T / dK^T come out with the head dimension on the TMEM lanes; each thread adds its 64 values
+// into fp32 accumulation buffers with coalesced red.global.add.f32 (several query blocks read the
+// same KV block), and a second kernel rounds those buffers to bf16.  This first version is one CTA
+// per unit, single-buffered, every step in sequence: correctness and the operand layouts first.
+#include <cuda.h>
+
+#include "bf1_common.cuh"
+
+namespace bf1 {
+
+constexpr int kBwdD = 128;
+constexpr int kBlock64 = 64;     // b: tokens per block
+constexpr int kBwdThreads = 128;
+
+struct BwdArgs {
+    const int32_t* cu_seqlens;
+    const int32_t* qb_seq;
+    const int32_t* qb_block;
+    const int32_t* kv_count;
+    const int32_t* kv_idx;
+    const int32_t* num_qblocks;
+    int32_t max_degree, capacity, total_tokens, hq, hkv;
+    int32_t* status;
+    float scale, scale_log2;
+    const __nv_bfloat16* o;
+    const __nv_bfloat16* d_o;
+    const float* lse;
+    __nv_bfloat16* dq;
+    float* dk32;   // [T, hkv, d] fp32 accumulation
+    float* dv32;
+};
+
+struct BwdSmem {
+    static constexpr int kQ = 0;                     // Q tile   [2 chunks][128 rows][128 B]
+    static constexpr int kDO = kQ + 32768;           // dO tile  same layout
+    static constexpr int kK = kDO + 32768;           // K tile   [2 chunks][64 rows][128 B]
+    static constexpr int kV = kK + 16384;            // V tile
+    static constexpr int kP = kV + 16384;            // P  [128 q rows][64 kv] bf16, 128-byte rows, swizzled
+    static constexpr int kDS = kP + 16384;           // dS same layout
+    static constexpr int kBar = kDS + 16384;
+    static constexpr int kTotal = kBar + 64;
+};
+
+__global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                               const __grid_constant__ CUtensorMap tm_k,
+                                                               const __grid_constant__ CUtensorMap tm_v,
+                                                               const __grid_constant__ CUtensorMap tm_do,
+                                                               const BwdArgs a) {
+    constexpr int D = kBwdD;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int slot = blockIdx.x, kvh = blockIdx.y;
+    if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
+    if (slot >= min(*a.num_qblocks, a.capacity)) return;
+    const int seq = a.qb_seq[slot], j = a.qb_block[slot];
+    const int cnt = min(max(a.kv_count[slot], 1), a.max_degree);
+    const int32_t* list = a.kv_idx + (size_t)slot * a.max_degree;
+    const int seq0 = a.cu_seqlens[seq];
+    const int seqlen = a.cu_seqlens[seq + 1] - seq0;
+    const int rows_valid = min(kBlock64, seqlen - j * kBlock64);
+    const int tok0 = seq0 + j * kBlock64;
+
+    const uint32_t base = smem_u32(smem);
+    const uint32_t sQ = base + BwdSmem::kQ, sDO = base + BwdSmem::kDO, sK = base + BwdSmem::kK, sV = base + BwdSmem::kV;
+    const uint32_t sP = base + BwdSmem::kP, sDS = base + BwdSmem::kDS;
+    const uint32_t bar_q = base + BwdSmem::kBar, bar_kv = bar_q + 8, bar_a = bar_q + 16, bar_b = bar_q + 24;
+    if (tid == 0) {
+        s_abort = (base & 1023u) ? 1 : 0;
+        if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
+        mbar_init(bar_q, 1);
+        mbar_init(bar_kv, 1);
+        mbar_init(bar_a, 1);
+        mbar_init(bar_b, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&s_tmem), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    volatile int* abort_flag = &s_abort;
+    constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128, kColDVt = 256, kColDKt = 320;
+    const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+
+    // rows of this thread: head hl, token tl of the query block
+    const int hl = tid >> 6, tl = tid & 63;
+    const int h = kvh * 2 + hl;
+    const int tok = tok0 + tl;
+    const bool row_ok = tl < rows_valid;
+
+    if (tid == 0 && !s_abort) {
+        mbar_expect_tx(bar_q, 65536);
+        tma_load_4d(sQ, &tm_q, 0, tok0, kvh * 2, 0, bar_q);
+        tma_load_4d(sDO, &tm_do, 0, tok0, kvh * 2, 0, bar_q);
+    }
+    // D_i = <dO_i, O_i> and the row's LSE in the log2 domain
+    float Drow = 0.f, lse2 = 0.f;
+    if (row_ok) {
+        const uint4* op = reinterpret_cast<const uint4*>(a.o + ((size_t)tok * a.hq + h) * D);
+        const uint4* gp = reinterpret_cast<const uint4*>(a.d_o + ((size_t)tok * a.hq + h) * D);
+#pragma unroll 4
+        for (int c = 0; c < D / 8; ++c) {
+            const uint4 ov = op[c], gv = gp[c];
+            const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                Drow = fmaf(__uint_as_float(ow[e] << 16), __uint_as_float(gw[e] << 16), Drow);
+                Drow = fmaf(__uint_as_float(ow[e] & 0xffff0000u), __uint_as_float(gw[e] & 0xffff0000u), Drow);
+            }
+        }
+        lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
+    }
+    mbar_wait(bar_q, 0, abort_flag, a.status);
+
+    constexpr uint32_t kHi = desc_hi_sw128(1024);
+    constexpr uint32_t kIdS = idesc_bf16_f32_ab(64, false, false);     // S, dP: 128 x 64, A and B K-major
+    constexpr uint32_t kIdQ = idesc_bf16_f32_ab(D, false, true);       // dQ: 128 x 128, B (K tile) MN-major
+    constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);       // dV^T, dK^T: A and B MN-major
+
+    for (int it = 0; it < cnt; ++it) {
+        int p = list[it];
+        if (p < 0 || p > j || (it == cnt - 1) != (p == j)) {            // stay inside the sequence
+            if (tid == 0 && a.status) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+            p = (it == cnt - 1) ? j : 0;
+        }
+        const bool diag = (it == cnt - 1);
+        const int kv_valid = min(kBlock64, seqlen - p * kBlock64);      // key rows of this block inside the sequence
+        if (tid == 0) {
+            mbar_expect_tx(bar_kv, 32768);
+            tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
+            tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
+            mbar_wait(bar_kv, it & 1, abort_flag, a.status);
+            tc_fence_after();
+            // S = Q K^T and dP = dO V^T: 8 k-steps of 16 over d
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
+                if (kk == 0) {
+                    mma_ss_lohi<false>(tmem + kColS, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
+                    mma_ss_lohi<false>(tmem + kColDP, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
+                } else {
+                    mma_ss_lohi<true>(tmem + kColS, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
+                    mma_ss_lohi<true>(tmem + kColDP, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
+                }
+            }
+            mma_commit(bar_a);
+        }
+        __syncwarp();
+        mbar_wait(bar_a, it & 1, abort_flag, a.status);
+        tc_fence_after();
+
+        // ---- P and dS for this thread's row, 32 columns at a time, written as bf16 rows ------------
+        const uint32_t prow = sP + tid * 128, dsrow = sDS + tid * 128;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t sr[32], dr[32];
+            tmem_ld32(t_lane + kColS + half * 32, sr);
+            tmem_ld32(t_lane + kColDP + half * 32, dr);
+            tmem_wait_ld();
+            uint32_t pw[16], dw[16];
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+                float pv[2], dv[2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int col = half * 32 + c + e;
+                    const bool on = row_ok && (!diag || col <= tl);   // causal triangle on the self block; no rows past the end
+                    const float pe = on ? ex2_approx(fmaf(__uint_as_float(sr[c + e]), a.scale_log2, -lse2)) : 0.f;
+                    pv[e] = pe;
+                    dv[e] = on ? pe * (__uint_as_float(dr[c + e]) - Drow) * a.scale : 0.f;
+                }
+                pw[c / 2] = pack_bf16x2(pv[0], pv[1]);
+                dw[c / 2] = pack_bf16x2(dv[0], dv[1]);
+            }
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk half * 4 + c4 of the 128-byte row
+                const int ch = (half * 4 + c4) ^ (tid & 7);
+                st_shared_v4(prow + (ch << 4), pw[4 * c4], pw[4 * c4 + 1], pw[4 * c4 + 2], pw[4 * c4 + 3]);
+                st_shared_v4(dsrow + (ch << 4), dw[4 * c4], dw[4 * c4 + 1], dw[4 * c4 + 2], dw[4 * c4 + 3]);
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+
+        if (tid == 0) {
+            tc_fence_after();
+            // dQ += dS K: A = dS [128 q][64 kv] K-major (4 k-steps of 16 kv = 32 bytes), B = K tile MN-major
+            // (16 kv rows = 2048 bytes per step, next 64 d columns 8 KB away)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const uint32_t alo = desc_lo_sw128(sDS, 16) + ((kk * 32) >> 4);
+                const uint32_t blo = desc_lo_sw128(sK, 8192) + ((kk * 2048) >> 4);
+                if (it == 0 && kk == 0) mma_ss_lohi<false>(tmem + kColDQ, alo, blo, kHi, kIdQ);
+                else mma_ss_lohi<true>(tmem + kColDQ, alo, blo, kHi, kIdQ);
+            }
+            // dV^T = dO^T P and dK^T = Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
+            // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t ko = (kk * 2048) >> 4;
+                if (kk == 0) {
+                    mma_ss_lohi<false>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                    mma_ss_lohi<false>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                } else {
+                    mma_ss_lohi<true>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                    mma_ss_lohi<true>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                }
+            }
+            mma_commit(bar_b);
+        }
+        __syncwarp();
+        mbar_wait(bar_b, it & 1, abort_flag, a.status);
+        tc_fence_after();
+
+        // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns -----------------
+        float* dvp = a.dv32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
+        float* dkp = a.dk32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
+        const size_t rstride = (size_t)a.hkv * D;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t vr[32], kr[32];
+            tmem_ld32(t_lane + kColDVt + half * 32, vr);
+            tmem_ld32(t_lane + kColDKt + half * 32, kr);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const int kvr = half * 32 + c;
+                if (kvr < kv_valid) {
+                    atomicAdd(dvp + kvr * rstride, __uint_as_float(vr[c]));
+                    atomicAdd(dkp + kvr * rstride, __uint_as_float(kr[c]));
+                }
+            }
+        }
+        tc_fence_before();
+        __syncthreads();   // K/V, P/dS buffers and the S/dP/dV^T/dK^T columns are free again
+    }
+
+    // ---- dQ rows -----------------------------------------------------------------------------------
+    tc_fence_after();
+    __nv_bfloat16* dqrow = a.dq + ((size_t)tok * a.hq + h) * D;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_lane + kColDQ + c * 32, r);
+        tmem_wait_ld();
+        if (row_ok) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 8) {
+                uint4 w;
+                w.x = pack_bf16x2(__uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
+                w.y = pack_bf16x2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                w.z = pack_bf16x2(__uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
+                w.w = pack_bf16x2(__uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
+                *reinterpret_cast<uint4*>(dqrow + c * 32 + e) = w;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// fp32 accumulation buffers -> bf16 gradients
+__global__ void bwd_round_kernel(const float* __restrict__ src_k, const float* __restrict__ src_v,
+                                 __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        dk[i] = __float2bfloat16_rn(src_k[i]);
+        dv[i] = __float2bfloat16_rn(src_v[i]);
+    }
+}
+
+int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box);   // bf1_attn.cu
+
+}  // namespace bf1
+
+using namespace bf1;
+
+extern "C" int64_t bf1_attn_bwd_workspace_bytes(int64_t total_tokens, int32_t hkv, int32_t d) {
+    if (total_tokens < 0 || hkv <= 0 || d <= 0) return -1;
+    return 2 * total_tokens * hkv * d * (int64_t)sizeof(float);
+}
+
+extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse,
+                            const void* d_o, const int32_t* cu_seqlens_dev, int32_t batch, int64_t total_tokens,
+                            int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d, float softmax_scale,
+                            const bf1_route* route, void* workspace, void* dq, void* dk, void* dv, void* stream) {
+    if (!q || !k || !v || !o || !lse || !d_o || !cu_seqlens_dev || !route || !workspace || !dq || !dk || !dv)
+        return fail(BF1_ERR_INVALID_ARG, "a pointer is null");
+    if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || hq <= 0 || hkv <= 0)
+        return fail(BF1_ERR_INVALID_ARG, "negative or zero size argument");
+    if (total_tokens > 0x7fffffffLL - 64) return fail(BF1_ERR_UNSUPPORTED, "total_tokens does not fit 32-bit token indices");
+    if (hq % hkv != 0) return fail(BF1_ERR_INVALID_ARG, "hq %d is not a multiple of hkv %d", hq, hkv);
+    if (hq / hkv != 2) return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 is supported", hq / hkv);
+    if (d != 128) return fail(BF1_ERR_UNSUPPORTED, "backward: head dimension %d: only 128 is supported", d);
+    if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o | (uintptr_t)d_o | (uintptr_t)dq | (uintptr_t)dk |
+         (uintptr_t)dv | (uintptr_t)workspace) & 15)
+        return fail(BF1_ERR_INVALID_ARG, "tensors and workspace must be 16-byte aligned");
+    if (!route->qb_seq || !route->qb_block || !route->kv_count || !route->kv_idx || !route->num_qblocks || !route->status)
+        return fail(BF1_ERR_INVALID_ARG, "a route array pointer is null");
+    if (route->capacity_qblocks < 1 || route->max_degree < 1 || hkv > 65535)
+        return fail(BF1_ERR_CAPACITY, "bad route capacities or hkv");
+    if (total_tokens == 0 || batch == 0) return BF1_OK;
+    int dev = 0, major = 0;
+    BF1_CUDA_CHECK(cudaGetDevice(&dev));
+    BF1_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major != 10) return fail(BF1_ERR_NO_DEVICE, "device compute capability %d.x is not sm_100", major);
+    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem::kTotal));
+    CUtensorMap tq, tk, tv, tg;
+    if (int rc = make_map_4d(&tq, q, total_tokens, hq, d, 2)) return rc;
+    if (int rc = make_map_4d(&tg, d_o, total_tokens, hq, d, 2)) return rc;
+    if (int rc = make_map_4d(&tk, k, total_tokens, hkv, d, 1)) return rc;
+    if (int rc = make_map_4d(&tv, v, total_tokens, hkv, d, 1)) return rc;
+    const size_t n_kv = (size_t)total_tokens * hkv * d;
+    BwdArgs a;
+    a.cu_seqlens = cu_seqlens_dev;
+    a.qb_seq = route->qb_seq;
+    a.qb_block = route->qb_block;
+    a.kv_count = route->kv_count;
+    a.kv_idx = route->kv_idx;
+    a.num_qblocks = route->num_qblocks;
+    a.max_degree = route->max_degree;
+    a.capacity = route->capacity_qblocks;
+    a.total_tokens = (int32_t)total_tokens;
+    a.hq = hq;
+    a.hkv = hkv;
+    a.status = route->status;
+    a.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
+    a.scale_log2 = a.scale * 1.4426950408889634f;
+    a.o = (const __nv_bfloat16*)o;
+    a.d_o = (const __nv_bfloat16*)d_o;
+    a.lse = lse;
+    a.dq = (__nv_bfloat16*)dq;
+    a.dk32 = (float*)workspace;
+    a.dv32 = a.dk32 + n_kv;
+    cudaStream_t st = (cudaStream_t)stream;
+    BF1_CUDA_CHECK(cudaMemsetAsync(workspace, 0, 2 * n_kv * sizeof(float), st));
+    dim3 grid(route->capacity_qblocks, hkv);
+    attn_bwd_kernel<<<grid, kBwdThreads, BwdSmem::kTotal, st>>>(tq, tk, tv, tg, a);
+    BF1_CUDA_CHECK(cudaGetLastError());
+    bwd_round_kernel<<<296, 512, 0, st>>>(a.dk32, a.dv32, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_kv);
+    BF1_CUDA_CHECK(cudaGetLastError());
+    return BF1_OK;
+}

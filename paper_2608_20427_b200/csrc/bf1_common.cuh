@@ -286,6 +286,11 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int n, bool b_mn_major) {
            | (static_cast<uint32_t>(128 >> 4) << 24);
 }
 
+// Same with a choice of major-ness for A as well (A from shared memory only).
+__host__ __device__ constexpr uint32_t idesc_bf16_f32_ab(int n, bool a_mn_major, bool b_mn_major) {
+    return idesc_bf16_f32(n, b_mn_major) | ((a_mn_major ? 1u : 0u) << 15);
+}
+
 // 32 lanes x 32 columns of 32-bit TMEM cells: thread i of the warp gets lane (base lane + i).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
