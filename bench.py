@@ -330,7 +330,15 @@ def run_single(args):
     lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
     work = torch.zeros(4, dtype=torch.int32, device=dev)
-    if args.mode == "dense":
+    if args.mode == "bwd":
+        d_o = torch.randn(q.shape, generator=torch.Generator(device=dev).manual_seed(w.seed), device=dev,
+                          dtype=torch.float32).to(torch.bfloat16)
+        bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
+        ws = torch.empty(int(bf1.load().bf1_attn_bwd_workspace_bytes(w.total_tokens, w.hkv, w.d)), dtype=torch.uint8,
+                         device=dev)
+        f = lambda: bf1.attn_bwd(q, k, v, o, lse, d_o, cu, w.max_seqlen, route, workspace=ws)
+        pairs = int(2.5 * sum(selected_pairs(n) for n in w.seqlens))   # five MMA groups against the forward's two
+    elif args.mode == "dense":
         f = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse, work=work)
         pairs = sum(n * (n + 1) // 2 for n in w.seqlens)
     else:
@@ -501,7 +509,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--single", default=None, choices=sorted(I.WORKLOADS),
                     help="only time `--steps` launches of one workload (used for profiling)")
-    ap.add_argument("--mode", default="bf1", choices=["bf1", "dense", "decode"])
+    ap.add_argument("--mode", default="bf1", choices=["bf1", "dense", "decode", "bwd"])
     args = ap.parse_args()
     if args.single:
         run_single(args)

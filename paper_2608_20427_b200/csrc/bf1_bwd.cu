@@ -49,21 +49,23 @@ struct BwdSmem {
     static constexpr int kDO = kQ + 32768;           // dO tile  same layout
     static constexpr int kK = kDO + 32768;           // K tile   [2 chunks][64 rows][128 B]
     static constexpr int kV = kK + 16384;            // V tile
-    static constexpr int kP = kV + 16384;            // P  [128 q rows][64 kv] bf16, 128-byte rows, swizzled
+    static constexpr int kP = kV;                    // P  [128 q rows][64 kv] bf16, 128-byte rows, swizzled: takes
+                                                     // over V's buffer once dP = dO V^T has been computed
     static constexpr int kDS = kP + 16384;           // dS same layout
     static constexpr int kBar = kDS + 16384;
     static constexpr int kTotal = kBar + 64;
 };
 
-__global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q,
+__global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k,
                                                                const __grid_constant__ CUtensorMap tm_v,
                                                                const __grid_constant__ CUtensorMap tm_do,
                                                                const BwdArgs a) {
     constexpr int D = kBwdD;
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint32_t s_tmem;
-    __shared__ int s_abort;
+    // no static shared memory: it would cost a whole extra kilobyte and with it the second CTA per SM
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + BwdSmem::kBar + 32);
+    int& s_abort = *reinterpret_cast<int*>(smem + BwdSmem::kBar + 36);
     const int tid = threadIdx.x, warp = tid >> 5;
     const int slot = blockIdx.x, kvh = blockIdx.y;
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     }
     __syncwarp();
     if (warp == 0) {
-        tmem_alloc(smem_u32(&s_tmem), 512);
+        tmem_alloc(smem_u32(&s_tmem), 256);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -99,7 +101,9 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* abort_flag = &s_abort;
-    constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128, kColDVt = 256, kColDKt = 320;
+    // dV^T and dK^T reuse the columns of S and dP (which the threads have turned into P and dS by then):
+    // 256 columns and 112 KB of shared memory per CTA let two CTAs share an SM
+    constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128, kColDVt = kColS, kColDKt = kColDP;
     const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
 
     // rows of this thread: head hl, token tl of the query block
@@ -278,7 +282,7 @@ __global__ void __launch_bounds__(kBwdThreads) attn_bwd_kernel(const __grid_cons
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 512);
+    if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
 // fp32 accumulation buffers -> bf16 gradients
@@ -326,6 +330,9 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     BF1_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
     if (major != 10) return fail(BF1_ERR_NO_DEVICE, "device compute capability %d.x is not sm_100", major);
     BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem::kTotal));
+    // two CTAs per SM need the whole shared-memory carve-out
+    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared));
     CUtensorMap tq, tk, tv, tg;
     if (int rc = make_map_4d(&tq, q, total_tokens, hq, d, 2)) return rc;
     if (int rc = make_map_4d(&tg, d_o, total_tokens, hq, d, 2)) return rc;
