@@ -141,18 +141,27 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
     constexpr uint32_t kIdQ = idesc_bf16_f32_ab(D, false, true);       // dQ: 128 x 128, B (K tile) MN-major
     constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);       // dV^T, dK^T: A and B MN-major
 
-    for (int it = 0; it < cnt; ++it) {
+    // list entry -> block index, kept inside the sequence whatever the list holds
+    auto entry = [&](int it) -> int {
         int p = list[it];
-        if (p < 0 || p > j || (it == cnt - 1) != (p == j)) {            // stay inside the sequence
+        if (p < 0 || p > j || (it == cnt - 1) != (p == j)) {
             if (tid == 0 && a.status) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
             p = (it == cnt - 1) ? j : 0;
         }
+        return p;
+    };
+    auto load_kv = [&](int p) {   // thread 0 only
+        mbar_expect_tx(bar_kv, 32768);
+        tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
+        tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
+    };
+    int p = entry(0);
+    if (tid == 0) load_kv(p);
+    for (int it = 0; it < cnt; ++it) {
+        const int p_next = (it + 1 < cnt) ? entry(it + 1) : 0;
         const bool diag = (it == cnt - 1);
         const int kv_valid = min(kBlock64, seqlen - p * kBlock64);      // key rows of this block inside the sequence
         if (tid == 0) {
-            mbar_expect_tx(bar_kv, 32768);
-            tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
-            tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
             mbar_wait(bar_kv, it & 1, abort_flag, a.status);
             tc_fence_after();
             // S = Q K^T and dP = dO V^T: 8 k-steps of 16 over d
@@ -236,6 +245,8 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
         __syncwarp();
         mbar_wait(bar_b, it & 1, abort_flag, a.status);
         tc_fence_after();
+        // K, V (and P, which lives in V's buffer) are free: fetch the next tile while the sums go out
+        if (tid == 0 && it + 1 < cnt) load_kv(p_next);
 
         // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns -----------------
         float* dvp = a.dv32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
@@ -257,7 +268,8 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
             }
         }
         tc_fence_before();
-        __syncthreads();   // K/V, P/dS buffers and the S/dP/dV^T/dK^T columns are free again
+        __syncthreads();   // dS buffer and the S/dP/dV^T/dK^T columns are free again
+        p = p_next;
     }
 
     // ---- dQ rows -----------------------------------------------------------------------------------
