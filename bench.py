@@ -226,6 +226,35 @@ def sweep(bf1, dev):
     return out
 
 
+def backward_sweep(bf1, dev):
+    """Backward over the same route (Section 4.2's gradient gate), one layer, 4K .. 32K: CUDA-event median of
+    10 calls (the call clears and rounds its fp32 dK/dV buffers: included).  FLOPs = 10 * d * pairs * Hq
+    (five MMA groups per block pair against the forward's two)."""
+    out = []
+    stream = torch.cuda.current_stream()
+    for name in ("qwen_4k", "qwen_8k", "qwen_16k", "qwen_32k"):
+        w = I.WORKLOADS[name]
+        q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+        d_o = torch.randn(q.shape, generator=torch.Generator(device=dev).manual_seed(w.seed), device=dev,
+                          dtype=torch.float32).to(torch.bfloat16)
+        cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+        route = bf1.plan_route(cu, w.max_seqlen)
+        o, lse = bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route)
+        ws = torch.empty(int(bf1.load().bf1_attn_bwd_workspace_bytes(w.total_tokens, w.hkv, w.d)), dtype=torch.uint8,
+                         device=dev)
+        f = lambda: bf1.attn_bwd(q, k, v, o, lse, d_o, cu, w.max_seqlen, route, workspace=ws)
+        for _ in range(3):
+            f()
+        ms = time_region(f, 10, stream)
+        route.check_status()
+        pairs = selected_pairs(w.seqlens[0])
+        tf = 10.0 * w.d * pairs * w.hq / ms / 1e9
+        out.append({"n": w.seqlens[0], "bwd_ms": round(ms, 4), "bwd_tflops": round(tf, 1),
+                    "frac_of_bf16_peak": round(tf / measured_peaks()["bf16_tflops"], 4)})
+        del q, k, v, d_o, o, lse, ws
+    return out
+
+
 def decode_sweep(bf1, dev):
     """Selected-page one-token decode (Section 5.4, Table 3's grid: 32K / 64K context, batch 1 / 8 / 32).
     A pool of 8192 physical pages (2.1 GB of K and V, far larger than L2) and 32 random page tables per
@@ -489,6 +518,7 @@ def run_ours(args):
     if not args.no_sweep and world == 1:
         line["sweep"] = sweep(bf1, dev)
         line["decode"] = decode_sweep(bf1, dev)
+        line["backward"] = backward_sweep(bf1, dev)
     if not args.no_cpu and world == 1:
         q, k, v = I.draw_qkv(w)
         val, dt, desc, thr = oracle_rate(w, q, k, v, target_s=15.0)
