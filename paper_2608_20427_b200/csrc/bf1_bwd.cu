@@ -184,26 +184,35 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
 
         // ---- P and dS for this thread's row, 32 columns at a time, written as bf16 rows ------------
         const uint32_t prow = sP + tid * 128, dsrow = sDS + tid * 128;
+        // masked entries get s = -inf (self block, warp-uniform branch) and rows past the end of the
+        // sequence an infinite LSE: both give P = 0 exactly, and with it dS = 0
+        const float lse_row = row_ok ? lse2 : INFINITY;
+        const uint64_t c2p = pack2(a.scale_log2, a.scale_log2), nlp = pack2(-lse_row, -lse_row);
+        const uint64_t scp = pack2(a.scale, a.scale), ndp = pack2(-Drow * a.scale, -Drow * a.scale);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             uint32_t sr[32], dr[32];
             tmem_ld32(t_lane + kColS + half * 32, sr);
             tmem_ld32(t_lane + kColDP + half * 32, dr);
             tmem_wait_ld();
+            if (diag) {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    if (half * 32 + c > tl) sr[c] = 0xff800000u;   // -inf: causal triangle
+            }
             uint32_t pw[16], dw[16];
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-                float pv[2], dv[2];
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int col = half * 32 + c + e;
-                    const bool on = row_ok && (!diag || col <= tl);   // causal triangle on the self block; no rows past the end
-                    const float pe = on ? ex2_approx(fmaf(__uint_as_float(sr[c + e]), a.scale_log2, -lse2)) : 0.f;
-                    pv[e] = pe;
-                    dv[e] = on ? pe * (__uint_as_float(dr[c + e]) - Drow) * a.scale : 0.f;
-                }
-                pw[c / 2] = pack_bf16x2(pv[0], pv[1]);
-                dw[c / 2] = pack_bf16x2(dv[0], dv[1]);
+            for (int c = 0; c < 16; ++c) {
+                const uint64_t x = fma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), c2p, nlp);
+                float x0, x1;
+                unpack2(x, x0, x1);
+                const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                // dS = P * (dP - D) * scale
+                const uint64_t t = fma2(pack2(__uint_as_float(dr[2 * c]), __uint_as_float(dr[2 * c + 1])), scp, ndp);
+                float d0, d1;
+                unpack2(mul2(pack2(p0, p1), t), d0, d1);
+                pw[c] = pack_bf16x2(p0, p1);
+                dw[c] = pack_bf16x2(d0, d1);
             }
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk half * 4 + c4 of the 128-byte row
