@@ -520,10 +520,21 @@ def run_ours(args):
         line["decode"] = decode_sweep(bf1, dev)
         line["backward"] = backward_sweep(bf1, dev)
     if not args.no_cpu and world == 1:
-        q, k, v = I.draw_qkv(w)
-        val, dt, desc, thr = oracle_rate(w, q, k, v, target_s=15.0)
-        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc,
-                                "seconds": dt}
+        # the oracle, as it stands, on the host cores: whole layers of the same step (every row),
+        # as many of the eight as fit in about 12 s (at least one, at most all eight)
+        from oracle import bf1_oracle as O
+        ocfg = O.cfg(w.block, w.local_blocks, w.global_first, w.dyadic)
+        t_cpu, layers_done = 0.0, 0
+        while layers_done < LAYERS and (layers_done == 0 or t_cpu * (layers_done + 1) / layers_done < 14.0):
+            q, k, v = (t.contiguous() for t in host[layers_done])
+            t0 = time.perf_counter()
+            O.attn_route(ocfg, q, k, v, w.cu_seqlens())
+            t_cpu += time.perf_counter() - t0
+            layers_done += 1
+        line["cpu_baseline"] = {"value": layers_done * layer_flops / t_cpu / 1e12, "unit": UNIT, "cores": O.threads(),
+                                "kind": "oracle", "seconds": t_cpu,
+                                "sample": "%d of the step's %d layers, every token row (%s, fp32 oracle)" % (
+                                    layers_done, LAYERS, w.name)}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -21,9 +21,9 @@
 //   warp 1      MMA issuer for S = Q K^T: runs up to two tiles ahead of the softmax (two S buffers),
 //   warp 3      MMA issuer for O += P V: a separate warp, so that neither kind of MMA waits behind
 //               a burst of the other while the tensor pipe's queue is full,
-//   warp 2      scheduler: fetches the next unit, decodes it, reads (and range-checks) its list,
-//               prefetches its Q/K/V blocks into L2 and queues it for the producer -- all of it
-//               global-memory latency that must not sit in front of the copies,
+//   warp 2      scheduler: fetches the next unit, decodes it, reads (and range-checks) its list
+//               and queues it for the producer -- all of it global-memory latency that must not
+//               sit in front of the copies,
 //   warps 4-7   softmax, one thread per tile row,
 //   warps 8-11  epilogue: take the finished O out of tensor memory, normalise, store O and LSE,
 //               while the softmax warps are already on the next unit.
@@ -48,7 +48,9 @@ static_assert(kRegsCtl + kRegsSoftmax + kRegsEpilogue <= 240, "register budgets 
 #ifndef BF1_PREFETCH_MODE
 #define BF1_PREFETCH_MODE 0
 #endif
-constexpr int kPrefetchMode = BF1_PREFETCH_MODE;   // L2 prefetch of queued units: 0 none, 1 Q only, 2 Q + K/V
+// TMA prefetch of queued units into L2 (0 none, 1 Q only, 2 Q + K/V).  Measured at 32K: mode 2 costs
+// 10 % (the prefetches queue in front of the real copies in the same TMA unit), mode 1 costs 1 %.
+constexpr int kPrefetchMode = BF1_PREFETCH_MODE;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row
                                             // maximum grows by more than 2^8
 
