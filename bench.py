@@ -226,6 +226,40 @@ def sweep(bf1, dev):
     return out
 
 
+def topology_sweep(bf1, dev):
+    """Does the route's topology change the kernel's cost?  (Section 5.1: equal-pair-count BF1, sliding and
+    static-random routes have nearly identical sparse kernel time.)  One 32K layer through routes with about
+    the same number of block pairs: BF1, a sliding window with the closest pair count, BF1 without block 0,
+    dyadic predecessors without a local window.  Reported per executed tile so that small differences in
+    the pair budget cancel."""
+    w = I.WORKLOADS["qwen_32k"]
+    n = w.seqlens[0]
+    q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+    cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+    o = torch.empty_like(q)
+    lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    nb = n // 64
+    target = sum(degree(j) for j in range(nb))
+    best_w = min(range(1, 64), key=lambda ww: abs(sum(min(j, ww) + 1 for j in range(nb)) - target))
+    routes = [("bf1", bf1.RouteCfg()), ("sliding W=%d (equal block-pair budget)" % best_w,
+                                        bf1.RouteCfg(local_blocks=best_w, global_first=0, dyadic=0)),
+              ("bf1 without block 0", bf1.RouteCfg(global_first=0)),
+              ("dyadic only (W=0)", bf1.RouteCfg(local_blocks=0, global_first=0, dyadic=1))]
+    out = []
+    for name, cfg in routes:
+        route = bf1.plan_route(cu, n, cfg)
+        f = lambda: bf1.attn_fwd(q, k, v, cu, n, route, out=o, lse=lse)
+        for _ in range(5):
+            f()
+        ms = time_region(f, 30, stream)
+        route.check_status()
+        tiles = int(route.kv_count[:nb].sum().item()) * w.hkv
+        out.append({"route": name, "block_pairs": tiles // w.hkv, "ms": round(ms, 5),
+                    "ns_per_tile_per_sm": round(ms * 1e6 / (tiles / 148.0), 1)})
+    return out
+
+
 def backward_sweep(bf1, dev):
     """Backward over the same route (Section 4.2's gradient gate), one layer, 4K .. 32K: CUDA-event median of
     10 calls (the call clears and rounds its fp32 dK/dV buffers: included).  FLOPs = 10 * d * pairs * Hq
@@ -519,6 +553,7 @@ def run_ours(args):
         line["sweep"] = sweep(bf1, dev)
         line["decode"] = decode_sweep(bf1, dev)
         line["backward"] = backward_sweep(bf1, dev)
+        line["topology"] = topology_sweep(bf1, dev)
     if not args.no_cpu and world == 1:
         # the oracle, as it stands, on the host cores: whole layers of the same step (every row),
         # as many of the eight as fit in about 12 s (at least one, at most all eight)
