@@ -37,7 +37,13 @@ namespace bf1 {
 constexpr int kBlock = 64;            // b: tokens per block
 constexpr int kRows = 128;            // MMA M: 2 query heads x 64 tokens
 constexpr int kThreads = 384;         // 12 warps
-constexpr int kQueue = 3;             // decoded units queued between scheduler and producer
+#ifndef BF1_QUEUE
+#define BF1_QUEUE 1
+#endif
+// Decoded units queued between scheduler and producer.  One is enough to hide the decode, and every
+// unit a CTA holds in advance is a unit another CTA cannot take at the end of the launch: with three
+// the last CTAs finished 20 us after the first at 32K, and 8K was 7 % slower.
+constexpr int kQueue = BF1_QUEUE;
 #ifndef BF1_REGS_CTL
 #define BF1_REGS_CTL 40
 #define BF1_REGS_SOFTMAX 144
@@ -114,6 +120,12 @@ struct Cfg {
 // Optional event trace (compiled in with -DBF1_TRACE only): per traced CTA and role, a list of
 // (event code << 32 | index, clock64) pairs, for reading the pipeline's timeline off-line.
 #ifdef BF1_TRACE
+__device__ long long* g_span_buf = nullptr;   // [grid][2] globaltimer at CTA entry / exit
+__device__ __forceinline__ long long globaltimer_ns() {
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ long long* g_trace_buf = nullptr;
 __device__ int g_trace_cap = 0;
 constexpr int kTraceCtas = 8;
@@ -242,6 +254,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     int* s_nqb = reinterpret_cast<int*>(smem + C::kMiscOff + 8);
 
 #ifdef BF1_TRACE
+    if (tid == 0 && g_span_buf) g_span_buf[2 * blockIdx.x] = globaltimer_ns();
     Tracer tr_cta;
     if (tid == 32) {   // lane 0 of the MMA warp: shares that role's trace area
         tr_cta.init(1);
@@ -759,6 +772,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     __syncthreads();
 #ifdef BF1_TRACE
     if (tid == 32) TR(tr_cta, 42, 0);
+    if (tid == 0 && g_span_buf) g_span_buf[2 * blockIdx.x + 1] = globaltimer_ns();
 #endif
     if (warp == 1) tmem_dealloc(tmem, C::kTmemCols);
     retire();
@@ -922,6 +936,10 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
 }  // namespace bf1
 
 #ifdef BF1_TRACE
+extern "C" int bf1_trace_span_set(long long* buf_dev) {
+    cudaMemcpyToSymbol(bf1::g_span_buf, &buf_dev, sizeof buf_dev);
+    return (int)cudaGetLastError();
+}
 extern "C" int bf1_trace_set(long long* buf_dev, int cap) {
     cudaMemcpyToSymbol(bf1::g_trace_buf, &buf_dev, sizeof buf_dev);
     cudaMemcpyToSymbol(bf1::g_trace_cap, &cap, sizeof cap);
