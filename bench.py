@@ -494,24 +494,50 @@ def run_ours(args):
     h2d = sum(t.numel() * t.element_size() for h in host for t in h)
     d2h = sum(t.numel() * t.element_size() for t in o_host + l_host)
 
-    def e2e_step():
+    # three streams: host->device copies, kernels, device->host copies; a layer's kernel waits for its
+    # inputs, its read-back waits for the kernel, and the next step's upload of a layer waits until the
+    # previous kernel on those buffers is done.  The two copy directions and the kernels overlap.
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    ev_in = [torch.cuda.Event() for _ in range(LAYERS)]
+    ev_k = [torch.cuda.Event() for _ in range(LAYERS)]
+    ev_out = [torch.cuda.Event() for _ in range(LAYERS)]
+
+    def e2e_step(first=False):
         bf1.plan_route(cu, n, route=route)
         for layer in range(LAYERS):
-            for src, dst in zip(host[layer], devb[layer]):
-                dst.copy_(src, non_blocking=True)
+            with torch.cuda.stream(s_in):
+                if not first:
+                    s_in.wait_event(ev_k[layer])        # the previous step's kernel has read these buffers
+                for src, dst in zip(host[layer], devb[layer]):
+                    dst.copy_(src, non_blocking=True)
+                ev_in[layer].record(s_in)
+            stream.wait_event(ev_in[layer])
+            if not first:
+                stream.wait_event(ev_out[layer])        # the previous step's read-back of these outputs is done
             q, k, v = devb[layer]
             bf1.attn_fwd(q, k, v, cu, n, route, out=outs[layer], lse=lses[layer])
-            o_host[layer].copy_(outs[layer], non_blocking=True)
-            l_host[layer].copy_(lses[layer], non_blocking=True)
+            ev_k[layer].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_k[layer])
+                o_host[layer].copy_(outs[layer], non_blocking=True)
+                l_host[layer].copy_(lses[layer], non_blocking=True)
+                ev_out[layer].record(s_out)
+
+    def e2e_join():
+        stream.wait_stream(s_in)
+        stream.wait_stream(s_out)
 
     e2e_steps = max(2, min(args.steps, 5))
-    e2e_step()
+    e2e_step(first=True)
+    e2e_join()
     barrier()
     e0.record(stream)
     for _ in range(e2e_steps):
         e2e_step()
+    e2e_join()
     e1.record(stream)
     barrier()
+    assert torch.equal(o_host[LAYERS - 1], outs[LAYERS - 1].cpu())   # the read-back really happened
     e2e_ms = e0.elapsed_time(e1)
     e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     e2e_value = whole_job_value(step_flops, e2e_ms / e2e_steps, world)
