@@ -2,7 +2,8 @@
 //
 // Work unit = one query block (64 tokens) of one sequence x one KV head.  The G = 2 query
 // heads that share the KV head are stacked into one M = 128 tile (rows 0..63: first head,
-// rows 64..127: second head), because they read the same K/V blocks through the same route
+// rows 64..127: second head; with G = 4 the tile is 4 heads x 32 tokens and a query block is two
+// units), because they read the same K/V blocks through the same route
 // list (the route is per block and the same for all heads, Section 3.1).  For every entry p
 // of the unit's list ("tile"):
 //   S = Q K[p]^T        tcgen05.mma, Q and K[p] in shared memory (TMA, 128-byte swizzle),
@@ -65,6 +66,8 @@ struct AttnArgs {
     int32_t batch;
     int32_t total_tokens;
     int32_t hq, hkv;
+    int32_t group;         // G = hq / hkv query heads per KV head: 2 or 4
+    int32_t r_shift;       // log2 of the tile rows per head R = 128 / G (6 or 5); a unit covers R query tokens
     float scale_log2;      // softmax scale * log2(e)
     int32_t dense;         // 1: every predecessor block, lists ignored
     // route (BF1 mode)
@@ -159,9 +162,15 @@ struct Unit {
 
 // Unit u of the hand-out order -> what to compute.  KV-head-major, so that the K/V of one
 // head stay hot in L2 while its query blocks are processed; inside a head longest list first.
+// With G = 4 the 128 tile rows are 4 heads x 32 tokens, so a 64-token query block is two units
+// (adjacent in the order: they read the same K/V blocks).  `kvh` carries the unit's token offset
+// inside its query block in its upper half.
 __device__ __forceinline__ void decode_unit(const AttnArgs& a, int nqb, int u, Unit& un) {
-    const int idx = u % nqb;
-    un.kvh = u / nqb;
+    const int halves = kBlock >> a.r_shift;
+    const int tok_off = (u % halves) << a.r_shift;
+    const int uq = u / halves;
+    const int idx = uq % nqb;
+    un.kvh = (uq / nqb) | (tok_off << 16);
     int seq, slot;
     if (!a.dense) {
         slot = a.order ? a.order[idx] : idx;
@@ -187,8 +196,8 @@ __device__ __forceinline__ void decode_unit(const AttnArgs& a, int nqb, int u, U
     }
     un.seq0 = a.cu_seqlens[seq];
     const int seqlen = a.cu_seqlens[seq + 1] - un.seq0;
-    un.rows_valid = min(kBlock, seqlen - un.j * kBlock);
-    un.tok0 = un.seq0 + un.j * kBlock;
+    un.rows_valid = max(0, min(1 << a.r_shift, seqlen - un.j * kBlock - tok_off));   // of this unit's R tokens
+    un.tok0 = un.seq0 + un.j * kBlock + tok_off;
 }
 
 template <int REGS>
@@ -330,7 +339,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             for (int s = 0; s < args.batch; ++s)
                 nqb0 += (args.cu_seqlens[s + 1] - args.cu_seqlens[s] + kBlock - 1) / kBlock;
         }
-        have0 = (int)blockIdx.x < nqb0 * args.hkv;
+        have0 = (int)blockIdx.x < nqb0 * args.hkv * (kBlock >> args.r_shift);
         if (have0) fetch_unit(blockIdx.x, nqb0, un0, my_p0);
     }
     if (warp == 1) {
@@ -343,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     const uint32_t tmem = *s_tmem_base;
     volatile int* abort_flag = s_abort;
     const int nqb = *s_nqb;
-    const int total_units = nqb * args.hkv;
+    const int total_units = nqb * args.hkv * (kBlock >> args.r_shift);
 #ifdef BF1_TRACE
     if (tid == 32) TR(tr_cta, 41, 0);
 #endif
@@ -365,12 +374,12 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                     if (have) fetch_unit(u, nqb, un, my_p);
                 }
                 if (have && kPrefetchMode >= 1) {
-                    if (lane == 0) tma_prefetch_l2_4d(&tm_q, 0, un.tok0, un.kvh * 2, 0);
+                    if (lane == 0) tma_prefetch_l2_4d(&tm_q, 0, un.tok0, (un.kvh & 0xffff) * args.group, 0);
                     if (kPrefetchMode >= 2 && lane < un.cnt) {
                         // pull this block into L2 ahead of the real load (needs no shared memory)
                         const int row = un.seq0 + my_p * kBlock;
-                        tma_prefetch_l2_4d(&tm_k, 0, row, un.kvh, 0);
-                        tma_prefetch_l2_4d(&tm_v, 0, row, un.kvh, 0);
+                        tma_prefetch_l2_4d(&tm_k, 0, row, un.kvh & 0xffff, 0);
+                        tma_prefetch_l2_4d(&tm_v, 0, row, un.kvh & 0xffff, 0);
                     }
                 }
                 const int qs = n % kQueue;
@@ -403,7 +412,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 mbar_wait(bar_sq_full + 8 * qs, (n / kQueue) & 1, abort_flag, args.status);
                 volatile QueueEntry* e = s_queue + qs;
                 int cnt = e->cnt;
-                const int rows_valid = e->rows_valid, tok0 = e->tok0, kvh = e->kvh, seq0 = e->seq0, j = e->j;
+                const int rows_valid = e->rows_valid, tok0 = e->tok0, kvh_packed = e->kvh, seq0 = e->seq0, j = e->j;
+                const int kvh = kvh_packed & 0xffff;
                 const int rslot = e->slot;
                 int my_p = e->p[lane];
                 if (*abort_flag) cnt = 0;
@@ -452,14 +462,14 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                             s_info[n & 1].x = cnt;
                             s_info[n & 1].y = rows_valid;
                             s_info[n & 1].z = tok0;
-                            s_info[n & 1].w = kvh;
+                            s_info[n & 1].w = kvh_packed;
                             mbar_arrive(bar_info + 8 * (n & 1));
                             if (cnt == 0) {
                                 mbar_arrive(bar_q_full);
                             } else {
                                 mbar_expect_tx(bar_q_full, C::kQBytes);
-                                // one copy: box = 64 elements x 64 tokens x 2 heads x all column chunks
-                                tma_load_4d(sQ, &tm_q, 0, tok0, kvh * 2, 0, bar_q_full);
+                                // one copy: box = 64 elements x R tokens x G heads x all column chunks
+                                tma_load_4d(sQ, &tm_q, 0, tok0, kvh * args.group, 0, bar_q_full);
                             }
                         }
                         __syncwarp();
@@ -582,8 +592,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         // ================================ softmax ==========================================
         setmaxnreg_inc<kRegsSoftmax>();
         const int quarter = warp & 3;                     // TMEM lanes this warp may touch
-        const int row = quarter * 32 + lane;              // tile row of this thread
-        const int tl = row & 63;                          // token inside the query block
+        const int row = quarter * 32 + lane;              // tile row of this thread: head row / R, token row % R
         const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const float c2 = args.scale_log2;
         uint32_t g = 0;
@@ -595,6 +604,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             TR(tr, 24, n);
             const int cnt = *abort_flag ? 0 : s_info[n & 1].x;
             const int rows_valid = s_info[n & 1].y, tok0 = s_info[n & 1].z, kvh = s_info[n & 1].w;
+            const int tl = (kvh >> 16) + (row & ((1 << args.r_shift) - 1));   // token inside the 64-token query block
             float m_used = 0.f;    // reference maximum (raw score units) the exponentials are taken against
             float l_run = 0.f;     // running sum of exp2((s - m_used) * c2)
             for (int i = 0; i < cnt; ++i, ++g) {
@@ -690,8 +700,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         setmaxnreg_dec<kRegsEpilogue>();
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        const int hl = row >> 6;                          // which head of the pair
-        const int tl = row & 63;
+        const int hl = row >> args.r_shift;               // which head of the group (uniform in a warp: R >= 32)
+        const int tl = row & ((1 << args.r_shift) - 1);   // token inside the unit
         const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const float c2 = args.scale_log2;
         for (int n = 0;; ++n) {
@@ -699,7 +709,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             volatile Handoff* h = s_hand + (n & 1);
             const float m_used = h->m[row], l_run = h->l[row];
             const int cnt = *abort_flag ? 0 : h->cnt;
-            const int rows_valid = h->rows_valid, tok0 = h->tok0, kvh = h->kvh;
+            const int rows_valid = h->rows_valid, tok0 = h->tok0, kvh = h->kvh & 0xffff;
             const uint32_t gl = (uint32_t)h->g_last;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_ho_free + 8 * (n & 1));
@@ -709,13 +719,13 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             const float inv_l = 1.f / l_run;
             const int tok = tok0 + tl;
             const bool store = tl < rows_valid;
-            __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * 2 + hl)) * D;
+            __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * args.group + hl)) * D;
             // Full blocks leave through shared memory and TMA stores: each warp packs 32 rows x 32
             // columns into its own 2 KB staging tile (64-byte swizzle, conflict-free) and one lane
             // hands it to the copy engine.  Scattered 16-byte global stores from here would sit in the
             // same load/store path as every other warp's mbarrier and shared-memory traffic and
             // slow the whole SM down.  16 columns at a time keeps the register budget small.
-            const bool full_tile = rows_valid == kBlock;   // warp-uniform
+            const bool full_tile = rows_valid == (1 << args.r_shift);   // warp-uniform
             const uint32_t stage_w = base + C::kStageOff + (warp & 3) * 2048;
             const uint32_t srow = stage_w + lane * 64;
 #pragma unroll
@@ -750,7 +760,8 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0) {
-                            tma_store_3d(&tm_o, (c >> 1) * 32, kvh * 2 + hl, tok0 + (quarter & 1) * 32, stage_w);
+                            tma_store_3d(&tm_o, (c >> 1) * 32, kvh * args.group + hl, tok0 + ((quarter * 32) & ((1 << args.r_shift) - 1)),
+                                         stage_w);
                             bulk_commit_group();
                         }
                     }
@@ -762,7 +773,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             }
             if (store) {
                 const float lse2 = m_used * c2 + lg2_approx(l_run);   // log2 domain
-                args.lse[(size_t)(kvh * 2 + hl) * args.total_tokens + tok] = lse2 * 0.6931471805599453f;
+                args.lse[(size_t)(kvh * args.group + hl) * args.total_tokens + tok] = lse2 * 0.6931471805599453f;
             }
         }
     }
@@ -802,12 +813,12 @@ static int get_encode_fn(EncodeTiledFn* fn) {
 // elements (128 bytes) x 64 tokens x `heads_per_box` heads x all chunks, 128-byte swizzle.  In shared
 // memory that is [chunk][head][token][128 B]: one K-major (or, for V, MN-major) 64-row tile per
 // chunk and head, which is what the MMA descriptors walk.
-static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box) {
+static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box, int tokens_per_box = kBlock) {
     EncodeTiledFn enc;
     if (int rc = get_encode_fn(&enc)) return rc;
     cuuint64_t dims[4] = {64, (cuuint64_t)T, (cuuint64_t)H, (cuuint64_t)(d / 64)};
     cuuint64_t strides[3] = {(cuuint64_t)H * d * 2, (cuuint64_t)d * 2, 128};
-    cuuint32_t box[4] = {64, (cuuint32_t)kBlock, (cuuint32_t)heads_per_box, (cuuint32_t)(d / 64)};
+    cuuint32_t box[4] = {64, (cuuint32_t)tokens_per_box, (cuuint32_t)heads_per_box, (cuuint32_t)(d / 64)};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -875,7 +886,9 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     if (total_tokens > 0x7fffffffLL - 64)
         return fail(BF1_ERR_UNSUPPORTED, "total_tokens %lld does not fit 32-bit token indices", (long long)total_tokens);
     if (hq % hkv != 0) return fail(BF1_ERR_INVALID_ARG, "hq %d is not a multiple of hkv %d", hq, hkv);
-    if (hq / hkv != 2) return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 is supported", hq / hkv);
+    const int group = hq / hkv;
+    if (group != 2 && group != 4)
+        return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 and G = 4 are supported", group);
     if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15)
         return fail(BF1_ERR_INVALID_ARG, "q, k, v and o must be 16-byte aligned");
@@ -890,14 +903,14 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     } else {
         slots = total_tokens / kBlock + batch;
     }
-    if (slots * hkv > 0x7fffffffLL) return fail(BF1_ERR_UNSUPPORTED, "too many work units");
+    if (slots * hkv * 2 > 0x7fffffffLL) return fail(BF1_ERR_UNSUPPORTED, "too many work units");
     if (total_tokens == 0 || batch == 0) return BF1_OK;   // nothing to do
     DeviceInfo info;
     if (int rc = device_info(&info)) return rc;
 
     CUtensorMap tq, tk, tv, to;
     if (int rc = make_store_map(&to, o, total_tokens, hq, d)) return rc;
-    if (int rc = make_map(&tq, q, total_tokens, hq, d, 2)) return rc;
+    if (int rc = make_map(&tq, q, total_tokens, hq, d, group, kRows / group)) return rc;
     if (int rc = make_map(&tk, k, total_tokens, hkv, d, 1)) return rc;
     if (int rc = make_map(&tv, v, total_tokens, hkv, d, 1)) return rc;
 
@@ -907,6 +920,8 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     a.total_tokens = (int32_t)total_tokens;
     a.hq = hq;
     a.hkv = hkv;
+    a.group = group;
+    a.r_shift = group == 2 ? 6 : 5;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
     a.scale_log2 = scale * 1.4426950408889634f;
     a.dense = route ? 0 : 1;
@@ -923,7 +938,7 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     a.o = reinterpret_cast<__nv_bfloat16*>(o);
     a.lse = lse;
 
-    const int64_t units = slots * hkv;
+    const int64_t units = slots * hkv * (group == 2 ? 1 : 2);
     const int grid = (int)(units < 2LL * info.sm_count ? units : 2LL * info.sm_count);
     if (d == 128)
         attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);

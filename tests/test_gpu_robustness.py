@@ -86,3 +86,19 @@ def test_large_scores_do_not_break_the_lazy_rescale():
         assert np.abs(lse - lse_ref).max() <= 1e-3 * max(1.0, np.abs(lse_ref).max())
         diff = o.astype(np.float64) - o_ref
         assert np.abs(diff).max() <= 4e-2 and np.sqrt((diff ** 2).mean() / (o_ref.astype(np.float64) ** 2).mean()) <= 1e-2
+
+
+@pytest.mark.parametrize("dense", [False, True], ids=["bf1", "dense"])
+@pytest.mark.parametrize("d", [64, 128])
+def test_group_of_four_query_heads(dense, d):
+    """G = 4 (e.g. 32 query / 8 KV heads): the tile is 4 heads x 32 tokens, a query block is two units."""
+    w = I.custom([1, 31, 32, 33, 64, 97, 1000, 2500], hq=8, hkv=2, d=d, seed=4500 + d)
+    q, k, v = I.draw_qkv(w)
+    o, lse, _ = run_gpu(w, q, k, v, dense=dense, guard=64)
+    if dense:
+        o_ref, lse_ref = O.dense_causal(q, k, v, w.cu_seqlens())
+    else:
+        o_ref, lse_ref = O.attn_route(oracle_cfg(w), q, k, v, w.cu_seqlens())
+    assert_parity(o, lse, o_ref, lse_ref)
+    for h in range(8):   # per head, so that a permuted head cannot hide in an average
+        assert np.abs(o[:, h] - o_ref[:, h]).max() <= 2e-2
