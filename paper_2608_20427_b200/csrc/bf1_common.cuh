@@ -106,16 +106,7 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
-// TMA: 3-D tiled load global -> shared, completion counted in bytes on an mbarrier.
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int c0, int c1, int c2,
-                                            uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-        : "memory");
-}
-// TMA: 4-D tiled load global -> shared.
+// TMA: 4-D tiled load global -> shared, completion counted in bytes on an mbarrier.
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int c0, int c1, int c2, int c3,
                                             uint32_t bar) {
     asm volatile(
@@ -124,17 +115,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int 
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
         : "memory");
 }
+// TMA prefetch of a tile into L2 only (no shared-memory destination, no completion signal).
 __device__ __forceinline__ void tma_prefetch_l2_4d(const void* tmap, int c0, int c1, int c2, int c3) {
     asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(
                      reinterpret_cast<uint64_t>(tmap)),
                  "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-// TMA prefetch of a tile into L2 only (no shared-memory destination, no completion signal).
-__device__ __forceinline__ void tma_prefetch_l2_3d(const void* tmap, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(
-                     reinterpret_cast<uint64_t>(tmap)),
-                 "r"(c0), "r"(c1), "r"(c2)
                  : "memory");
 }
 // TMA: 3-D tiled store shared -> global (bulk async group), and the group bookkeeping.
@@ -149,10 +134,6 @@ __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bul
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // all of this thread's bulk stores are complete
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// barrier among `count` threads (ids 1..15; 0 is __syncthreads)
-__device__ __forceinline__ void named_barrier(int id, int count) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -193,33 +174,9 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
                  : "memory");
 }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate.
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
-        "}\n" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc].
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
-        "}\n" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// The same two MMAs with the descriptors given as (low, high) 32-bit halves and the
-// accumulate flag known at compile time: the issuing thread is a single warp, so every
+// D[tmem] (+)= A * B, bf16 inputs, fp32 accumulate; A from shared memory (mma_ss_lohi) or tensor memory
+// (mma_ts_lohi), B from shared memory.  Descriptors are given as (low, high) 32-bit halves and the
+// accumulate flag is known at compile time: the issuing thread is a single warp, so every
 // instruction it spends on descriptor arithmetic delays the tensor pipe.
 template <bool kAccumulate>
 __device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
@@ -250,29 +207,20 @@ __device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, ui
         "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
         : "memory");
 }
-// Halves of the 128-byte-swizzle descriptor described below.
+// Shared-memory matrix descriptor for tcgen05.mma with 128-byte swizzle, as its two 32-bit halves.
+// The layout is the one TMA writes with CU_TENSOR_MAP_SWIZZLE_128B: 128-byte rows, 16-byte chunk
+// index XOR (row & 7), atoms of 8 rows = 1024 bytes, 1024-byte aligned.
+//   K-major operand (rows = M or N, 64 bf16 of K per 128-byte row): sbo = bytes between
+//   consecutive 8-row groups (1024), lbo unused.
+//   MN-major operand (rows = K, 64 bf16 of M or N per 128-byte row): sbo = bytes between
+//   consecutive 8-row (K) groups, lbo = bytes between consecutive 64-element chunks of M / N.
+// Low word: start address / 16 in bits 0..13, lbo / 16 in bits 16..29.  High word: sbo / 16 in bits
+// 0..13 (32..45 of the descriptor), descriptor version 1 (bit 46), SWIZZLE_128B (bits 61..63).
 __device__ __forceinline__ uint32_t desc_lo_sw128(uint32_t saddr, uint32_t lbo_bytes) {
     return ((saddr & 0x3FFFF) >> 4) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
 }
 __host__ __device__ constexpr uint32_t desc_hi_sw128(uint32_t sbo_bytes) {
-    return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14) | (2u << 29);   // version 1 (bit 46), SWIZZLE_128B (bits 61..63)
-}
-
-// Shared-memory matrix descriptor for tcgen05.mma, 128-byte swizzle (the layout TMA writes
-// with CU_TENSOR_MAP_SWIZZLE_128B: 128-byte rows, 16-byte chunk index XOR (row & 7), atoms
-// of 8 rows = 1024 bytes, 1024-byte aligned).
-//   K-major operand (rows = M or N, 64 bf16 of K per 128-byte row): sbo = bytes between
-//   consecutive 8-row groups (1024), lbo unused.
-//   MN-major operand (rows = K, 64 bf16 of N per 128-byte row): sbo = bytes between
-//   consecutive 8-row (K) groups, lbo = bytes between consecutive 64-element N chunks.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
-    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= 1ull << 46;  // descriptor version for sm_100
-    d |= 2ull << 61;  // SWIZZLE_128B
-    return d;
+    return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14) | (2u << 29);
 }
 
 // Instruction descriptor for kind::f16 with bf16 A/B and fp32 D, M = 128.
