@@ -218,11 +218,29 @@ def sweep(bf1, dev):
         ms_s, ms_d = statistics.median(meds["bf1"]), statistics.median(meds["dense"])
         n = w.seqlens[0]
         pairs = selected_pairs(n)
+        m = int(math.log2(n // 64))
+        closed = n * 64 * m - 64 * 64 * m + n * 65 // 2        # n log n total for n = 64 * 2^m (Prop. 1's accounting)
         out.append({"n": n, "bf1_ms": round(ms_s, 5), "dense_ms": round(ms_d, 5), "speedup": round(ms_d / ms_s, 3),
                     "bf1_tflops": round(flops(pairs, w.d, w.hq) / ms_s / 1e9, 1),
                     "dense_tflops": round(flops(n * (n + 1) // 2, w.d, w.hq) / ms_d / 1e9, 1),
+                    "selected_pairs_planner": int(route.total_pairs.item()), "selected_pairs_closed_form": closed,
                     "pair_reduction": round(n * (n + 1) / 2 / pairs, 3), "inputs": "L2-warm (same buffers re-run)"})
         del q, k, v, o, lse
+    # the ragged batch (3001, 8192, 12345, 16384 tokens) in one varlen launch
+    w = I.WORKLOADS["ragged"]
+    q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+    cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+    route = bf1.plan_route(cu, w.max_seqlen)
+    o = torch.empty_like(q)
+    lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
+    f = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
+    for _ in range(5):
+        f()
+    ms = time_region(f, 30, torch.cuda.current_stream())
+    pairs = sum(selected_pairs(x) for x in w.seqlens)
+    out.append({"ragged_seqlens": list(w.seqlens), "bf1_ms": round(ms, 5),
+                "bf1_tflops": round(flops(pairs, w.d, w.hq) / ms / 1e9, 1),
+                "selected_pairs_planner": int(route.total_pairs.item()), "selected_pairs_closed_form": pairs})
     return out
 
 
@@ -592,8 +610,14 @@ def run_ours(args):
             O.attn_route(ocfg, q, k, v, w.cu_seqlens())
             t_cpu += time.perf_counter() - t0
             layers_done += 1
+        cpu_model = ""
+        try:
+            with open("/proc/cpuinfo") as f:
+                cpu_model = next((ln.split(":", 1)[1].strip() for ln in f if ln.startswith("model name")), "")
+        except OSError:
+            pass
         line["cpu_baseline"] = {"value": layers_done * layer_flops / t_cpu / 1e12, "unit": UNIT, "cores": O.threads(),
-                                "kind": "oracle", "seconds": t_cpu,
+                                "kind": "oracle", "seconds": t_cpu, "cpu_model": cpu_model,
                                 "sample": "%d of the step's %d layers, every token row (%s, fp32 oracle)" % (
                                     layers_done, LAYERS, w.name)}
     print(json.dumps(line))
