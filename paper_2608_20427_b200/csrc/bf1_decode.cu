@@ -21,6 +21,7 @@ namespace bf1 {
 
 constexpr int kPage = 64;             // tokens per page = block width b
 constexpr int kDecThreads = 128;
+constexpr int kDecStages = 2;          // page-pair buffers per CTA in the one-CTA-per-list kernel (3 measured the same)
 
 struct DecodeArgs {
     const __nv_bfloat16* q;           // [batch, hq, d]
@@ -204,6 +205,140 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
     if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Large batches: one CTA per (sequence, KV head) walks the whole page list with an online softmax,
+// the next page pair streaming in (cp.async, kDecStages buffers) while the current one is used.  There are
+// enough CTAs to fill the GPU without splitting a list over CTAs, so the partial results, the
+// ticket and the combine of decode_kernel (three more trips to L2 per page) are not needed.
+template <int D>
+__global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeArgs a) {
+    constexpr int kRowWords = D / 2;
+    constexpr int kVecPerRow = D / 8;
+    constexpr int kVecPerThread = kPage * kVecPerRow / kDecThreads;
+    constexpr int kPageBytes = kPage * D * 2;
+    extern __shared__ __align__(16) uint8_t dsmem[];    // [stage][K | V][64 rows][D bf16], K chunks XOR-swizzled
+    __shared__ __align__(16) float sQ[2][D];
+    __shared__ __align__(16) float sP[2][kPage];
+    __shared__ float sRed[2][2];
+
+    const int kvh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
+    const int h = tid >> 6, r = tid & 63;
+    const int cnt = a.count[s];
+    const int n = a.seqlens[s];
+    if (cnt <= 0) return;
+    const int j = (n - 1) / kPage;
+    if (j != a.block[s]) {            // the plan belongs to another route epoch
+        if (tid == 0 && kvh == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+        return;
+    }
+    const int32_t* pages = a.page + (size_t)s * a.max_degree;
+    auto issue_page = [&](int e, int stage) {
+        int pg = pages[e];
+        if (pg < 0 || pg >= a.num_pages) {
+            if (tid == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+            pg = 0;
+        }
+        const size_t row_stride = (size_t)a.hkv * D;
+        const __nv_bfloat16* kp = a.k_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
+        const __nv_bfloat16* vp = a.v_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
+        const uint32_t kb = smem_u32(dsmem) + stage * 2 * kPageBytes, vb = kb + kPageBytes;
+#pragma unroll
+        for (int q = 0; q < kVecPerThread; ++q) {
+            const int i = tid + q * kDecThreads, rr = i / kVecPerRow, c = i % kVecPerRow;
+            cp_async16(kb + rr * (D * 2) + ((c ^ (rr & 7)) << 4), kp + rr * row_stride + c * 8);
+            cp_async16(vb + rr * (D * 2) + (c << 4), vp + rr * row_stride + c * 8);
+        }
+    };
+#pragma unroll
+    for (int e = 0; e < kDecStages - 1; ++e) {
+        if (e < cnt) issue_page(e, e);
+        cp_async_commit();                               // possibly empty: keeps the group count uniform
+    }
+    for (int i = tid; i < 2 * D; i += kDecThreads)
+        sQ[i / D][i % D] = __bfloat162float(a.q[((size_t)s * a.hq + kvh * 2 + i / D) * D + i % D]);
+
+    constexpr int kColsPerThread = D / 64;
+    const int c0 = r * kColsPerThread;
+    float m_run = -INFINITY, l_run = 0.f, acc[2] = {0.f, 0.f};
+    for (int e = 0; e < cnt; ++e) {
+        if (e + kDecStages - 1 < cnt) issue_page(e + kDecStages - 1, (e + kDecStages - 1) % kDecStages);
+        cp_async_commit();
+        cp_async_wait<kDecStages - 1>();                 // page e has landed (the younger groups may be in flight)
+        __syncthreads();
+        const int valid = (e == cnt - 1) ? (n - j * kPage) : kPage;   // self page: tokens up to n-1 only
+        const uint32_t(*sK)[kRowWords] = reinterpret_cast<const uint32_t(*)[kRowWords]>(dsmem + (e % kDecStages) * 2 * kPageBytes);
+        const uint32_t(*sV)[kRowWords] =
+            reinterpret_cast<const uint32_t(*)[kRowWords]>(dsmem + (e % kDecStages) * 2 * kPageBytes + kPageBytes);
+        float sc0 = 0.f, sc1 = 0.f;
+#pragma unroll
+        for (int c = 0; c < kVecPerRow; ++c) {
+            const uint4 kw = *reinterpret_cast<const uint4*>(&sK[r][(c ^ (r & 7)) * 4]);
+            const float4 qa = *reinterpret_cast<const float4*>(&sQ[h][c * 8]);
+            const float4 qb = *reinterpret_cast<const float4*>(&sQ[h][c * 8 + 4]);
+            sc0 = fmaf(qa.x, __uint_as_float(kw.x << 16), sc0);
+            sc1 = fmaf(qa.y, __uint_as_float(kw.x & 0xffff0000u), sc1);
+            sc0 = fmaf(qa.z, __uint_as_float(kw.y << 16), sc0);
+            sc1 = fmaf(qa.w, __uint_as_float(kw.y & 0xffff0000u), sc1);
+            sc0 = fmaf(qb.x, __uint_as_float(kw.z << 16), sc0);
+            sc1 = fmaf(qb.y, __uint_as_float(kw.z & 0xffff0000u), sc1);
+            sc0 = fmaf(qb.z, __uint_as_float(kw.w << 16), sc0);
+            sc1 = fmaf(qb.w, __uint_as_float(kw.w & 0xffff0000u), sc1);
+        }
+        const float sc = (r < valid) ? (sc0 + sc1) * a.scale_log2 : -INFINITY;   // log2 domain
+        float mx = sc;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = mx;
+        __syncthreads();
+        const float m_new = fmaxf(m_run, fmaxf(sRed[h][0], sRed[h][1]));   // finite: key 0 of every page is valid
+        const float alpha = exp2f(m_run - m_new);                           // 0 on the first page
+        const float p = exp2f(sc - m_new);
+        sP[h][r] = p;
+        float sum = p;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        __syncthreads();                                 // sRed reads done, sP written
+        if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = sum;
+        __syncthreads();
+        l_run = l_run * alpha + (sRed[h][0] + sRed[h][1]);
+        m_run = m_new;
+        acc[0] *= alpha;
+        acc[1] *= alpha;
+        if (kColsPerThread == 2) {
+            for (int k4 = 0; k4 < valid; k4 += 4) {      // never touch V rows past the newest token
+                const float4 pk = *reinterpret_cast<const float4*>(&sP[h][k4]);
+                const float pv[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    if (k4 + q4 < valid) {
+                        const uint32_t vw = sV[k4 + q4][r];
+                        acc[0] = fmaf(pv[q4], __uint_as_float(vw << 16), acc[0]);
+                        acc[1] = fmaf(pv[q4], __uint_as_float(vw & 0xffff0000u), acc[1]);
+                    }
+                }
+            }
+        } else {
+            const __nv_bfloat16* sVh = reinterpret_cast<const __nv_bfloat16*>(&sV[0][0]);
+#pragma unroll 8
+            for (int k = 0; k < valid; ++k) acc[0] = fmaf(sP[h][k], __bfloat162float(sVh[k * D + c0]), acc[0]);
+        }
+        __syncthreads();                                 // sP, sRed and this stage are free again
+    }
+    const float inv = 1.f / l_run;
+    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + kvh * 2 + h) * D;
+#pragma unroll
+    for (int c = 0; c < kColsPerThread; ++c) orow[c0 + c] = __float2bfloat16_rn(acc[c] * inv);
+    if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+}
+
 // One thread per sequence: Eq. 1 for the block of the newest token, mapped through the page table.
 __global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_table, int max_pages_per_seq,
                                    int batch, bf1_route_cfg cfg, bf1_decode_plan plan) {
@@ -316,9 +451,26 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
     a.o = (__nv_bfloat16*)o;
     a.lse = lse;
     a.batch = batch;
-    dim3 grid(plan->max_degree, hkv, batch);
-    if (d == 128) decode_kernel<128><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
-    else decode_kernel<64><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
+    static int sm_count[64] = {};
+    int dev = 0;
+    BF1_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return fail(BF1_ERR_NO_DEVICE, "device ordinal %d out of range", dev);
+    if (!sm_count[dev]) {
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 128 * 2));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 64 * 2));
+        BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+    }
+    if ((int64_t)batch * hkv >= sm_count[dev]) {
+        // enough (sequence, KV head) pairs to fill the GPU: one CTA walks a whole list
+        dim3 grid(hkv, batch);
+        if (d == 128) decode_fused_kernel<128><<<grid, kDecThreads, kDecStages * 2 * 64 * 128 * 2, (cudaStream_t)stream>>>(a);
+        else decode_fused_kernel<64><<<grid, kDecThreads, kDecStages * 2 * 64 * 64 * 2, (cudaStream_t)stream>>>(a);
+    } else {
+        // few pairs: split every list over CTAs (one page each) and combine
+        dim3 grid(plan->max_degree, hkv, batch);
+        if (d == 128) decode_kernel<128><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
+        else decode_kernel<64><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
+    }
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
 }

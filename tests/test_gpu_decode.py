@@ -100,6 +100,33 @@ def test_long_context_decode_32k_and_64k():
     check(w, q, k, v, out, lse, last)
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_large_batch_takes_the_one_cta_per_list_path(d):
+    """batch x KV heads >= number of SMs: one CTA walks a whole page list with an online softmax."""
+    rng = np.random.default_rng(7)
+    lens = [int(x) for x in rng.integers(1, 3000, size=40)] + [1, 64, 65, 0, 4097]
+    w = I.custom(lens, hq=8, hkv=4, d=d, seed=3500 + d)    # 45 x 4 = 180 pairs
+    q, k, v = I.draw_qkv(w)
+    k_pages, v_pages, table = paged_cache(w, k, v, seed=5)
+    out, lse, plan, last = run_decode(w, q, k_pages, v_pages, table)
+    assert int(plan.status.item()) == 0
+    check(w, q, k, v, out, lse, last)
+    # NaN behind the newest token and in unselected pages must not leak on this path either
+    used = set(int(x) for x in table.flatten().tolist() if x >= 0)
+    for pg in range(k_pages.shape[0]):
+        if pg not in used:
+            k_pages[pg] = float("nan")
+            v_pages[pg] = float("nan")
+    for s_, n_ in enumerate(w.seqlens):
+        if n_ % 64:
+            pg = int(table[s_, (n_ - 1) // 64])
+            k_pages[pg, n_ % 64:] = float("nan")
+            v_pages[pg, n_ % 64:] = float("nan")
+    out1, lse1, _, _ = run_decode(w, q, k_pages, v_pages, table)
+    live = [i for i, n_ in enumerate(lens) if n_ > 0]
+    assert np.array_equal(out[live], out1[live]) and np.array_equal(lse[:, live], lse1[:, live])
+
+
 def test_page_permutation_invariance_and_zero_decoy_leakage():
     w = I.custom([700, 3001], hq=4, hkv=2, d=128, seed=3200)
     q, k, v = I.draw_qkv(w)
