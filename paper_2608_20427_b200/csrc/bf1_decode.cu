@@ -21,7 +21,7 @@ namespace bf1 {
 
 constexpr int kPage = 64;             // tokens per page = block width b
 constexpr int kDecThreads = 128;
-constexpr int kDecStages = 2;          // page-pair buffers per CTA in the one-CTA-per-list kernel (3 measured the same)
+constexpr int kDecStages = 3;          // page-pair buffers per CTA in the one-CTA-per-list kernel
 
 struct DecodeArgs {
     const __nv_bfloat16* q;           // [batch, hq, d]
@@ -214,23 +214,45 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// Large batches: one CTA per (sequence, KV head) walks the whole page list with an online softmax,
-// the next page pair streaming in (cp.async, kDecStages buffers) while the current one is used.  There are
-// enough CTAs to fill the GPU without splitting a list over CTAs, so the partial results, the
-// ticket and the combine of decode_kernel (three more trips to L2 per page) are not needed.
+// cp.async that writes zeros when src_bytes is 0 (rows behind the newest token: unwritten cache memory
+// that may hold anything, NaN included, and must not reach a multiply)
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+
+// Large batches: one CTA per (sequence, KV head) walks the whole page list.  There are enough CTAs to
+// fill the GPU without splitting a list over CTAs, so the partial results, the ticket and the combine
+// of decode_kernel (three more trips to L2 per page) are not needed.  Pages stream in through a
+// kDecStages-deep cp.async ring with ONE block-wide synchronisation per page; inside a page each of the
+// four warps owns 16 keys and keeps its own online-softmax state (max, sum, O) for both grouped heads,
+// merged once at the end.  The arithmetic uses warp-level mma (m16n8k16: the two heads are rows 0 and 1
+// of the 16-row operand, the rest is zero): the work is memory-bound, but as scalar FMAs it was a chain
+// of 1500 dependent instructions and five synchronisations per page, which is what bounded the kernel.
 template <int D>
 __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeArgs a) {
-    constexpr int kRowWords = D / 2;
-    constexpr int kVecPerRow = D / 8;
+    constexpr int kRowBytes = D * 2;
+    constexpr int kVecPerRow = D / 8;                   // 16-byte chunks per row
     constexpr int kVecPerThread = kPage * kVecPerRow / kDecThreads;
     constexpr int kPageBytes = kPage * D * 2;
-    extern __shared__ __align__(16) uint8_t dsmem[];    // [stage][K | V][64 rows][D bf16], K chunks XOR-swizzled
-    __shared__ __align__(16) float sQ[2][D];
-    __shared__ __align__(16) float sP[2][kPage];
-    __shared__ float sRed[2][2];
+    // [stage][K | V][64 rows][D bf16]; the 16-byte chunks of every row are XOR-swizzled with (row & 7), which
+    // keeps both the B-fragment loads of K (8 rows, same chunk) and the ldmatrix rows of V conflict-free
+    extern __shared__ __align__(128) uint8_t dsmem[];
+    __shared__ float sM[4][2], sL[4][2];
+    __shared__ float sO[4][2][D];
 
     const int kvh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
-    const int h = tid >> 6, r = tid & 63;
+    const int warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int cnt = a.count[s];
     const int n = a.seqlens[s];
     if (cnt <= 0) return;
@@ -239,6 +261,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         if (tid == 0 && kvh == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
         return;
     }
+    const int tail = n - j * kPage;   // valid tokens of the self page (the last list entry)
     const int32_t* pages = a.page + (size_t)s * a.max_degree;
     auto issue_page = [&](int e, int stage) {
         int pg = pages[e];
@@ -246,6 +269,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
             if (tid == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
             pg = 0;
         }
+        const int valid = (e == cnt - 1) ? tail : kPage;
         const size_t row_stride = (size_t)a.hkv * D;
         const __nv_bfloat16* kp = a.k_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
         const __nv_bfloat16* vp = a.v_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
@@ -253,8 +277,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
 #pragma unroll
         for (int q = 0; q < kVecPerThread; ++q) {
             const int i = tid + q * kDecThreads, rr = i / kVecPerRow, c = i % kVecPerRow;
-            cp_async16(kb + rr * (D * 2) + ((c ^ (rr & 7)) << 4), kp + rr * row_stride + c * 8);
-            cp_async16(vb + rr * (D * 2) + (c << 4), vp + rr * row_stride + c * 8);
+            const uint32_t off = rr * kRowBytes + ((c ^ (rr & 7)) << 4);
+            const uint32_t nbytes = rr < valid ? 16u : 0u;
+            cp_async16_zfill(kb + off, kp + rr * row_stride + c * 8, nbytes);
+            cp_async16_zfill(vb + off, vp + rr * row_stride + c * 8, nbytes);
         }
     };
 #pragma unroll
@@ -262,81 +288,116 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         if (e < cnt) issue_page(e, e);
         cp_async_commit();                               // possibly empty: keeps the group count uniform
     }
-    for (int i = tid; i < 2 * D; i += kDecThreads)
-        sQ[i / D][i % D] = __bfloat162float(a.q[((size_t)s * a.hq + kvh * 2 + i / D) * D + i % D]);
+    // A fragments of Q: rows 0 and 1 of the 16-row operand are the two grouped heads, the rest zero
+    uint32_t qa[D / 16][2];
+    {
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + ((size_t)s * a.hq + kvh * 2 + (gid & 1)) * D);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+            qa[kk][0] = gid < 2 ? qrow[kk * 8 + tig] : 0u;          // columns kk*16 + 2*tig, +1
+            qa[kk][1] = gid < 2 ? qrow[kk * 8 + tig + 4] : 0u;      // columns kk*16 + 8 + 2*tig, +1
+        }
+    }
+    float m_run = -INFINITY, l_run = 0.f;                // per lane: head gid (lanes with gid >= 2 carry dummies)
+    float acc[D / 8][4];
+#pragma unroll
+    for (int dn = 0; dn < D / 8; ++dn) acc[dn][0] = acc[dn][1] = acc[dn][2] = acc[dn][3] = 0.f;
+    const int key0 = warp * 16;                          // this warp's 16 keys of every page
 
-    constexpr int kColsPerThread = D / 64;
-    const int c0 = r * kColsPerThread;
-    float m_run = -INFINITY, l_run = 0.f, acc[2] = {0.f, 0.f};
     for (int e = 0; e < cnt; ++e) {
+        cp_async_wait<kDecStages - 2>();                 // page e has landed (for this thread's copies)
+        __syncthreads();                                 // ... for everybody's; and page e-1 is no longer read
         if (e + kDecStages - 1 < cnt) issue_page(e + kDecStages - 1, (e + kDecStages - 1) % kDecStages);
         cp_async_commit();
-        cp_async_wait<kDecStages - 1>();                 // page e has landed (the younger groups may be in flight)
-        __syncthreads();
-        const int valid = (e == cnt - 1) ? (n - j * kPage) : kPage;   // self page: tokens up to n-1 only
-        const uint32_t(*sK)[kRowWords] = reinterpret_cast<const uint32_t(*)[kRowWords]>(dsmem + (e % kDecStages) * 2 * kPageBytes);
-        const uint32_t(*sV)[kRowWords] =
-            reinterpret_cast<const uint32_t(*)[kRowWords]>(dsmem + (e % kDecStages) * 2 * kPageBytes + kPageBytes);
-        float sc0 = 0.f, sc1 = 0.f;
+        const int valid = (e == cnt - 1) ? tail : kPage;
+        if (key0 >= valid) continue;                     // warp-uniform: none of this warp's keys exists
+        const uint32_t kb = smem_u32(dsmem) + (e % kDecStages) * 2 * kPageBytes, vb = kb + kPageBytes;
+        // ---- scores of 16 keys: two n-tiles of 8 keys, D / 16 k-steps ----------------------------
+        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-        for (int c = 0; c < kVecPerRow; ++c) {
-            const uint4 kw = *reinterpret_cast<const uint4*>(&sK[r][(c ^ (r & 7)) * 4]);
-            const float4 qa = *reinterpret_cast<const float4*>(&sQ[h][c * 8]);
-            const float4 qb = *reinterpret_cast<const float4*>(&sQ[h][c * 8 + 4]);
-            sc0 = fmaf(qa.x, __uint_as_float(kw.x << 16), sc0);
-            sc1 = fmaf(qa.y, __uint_as_float(kw.x & 0xffff0000u), sc1);
-            sc0 = fmaf(qa.z, __uint_as_float(kw.y << 16), sc0);
-            sc1 = fmaf(qa.w, __uint_as_float(kw.y & 0xffff0000u), sc1);
-            sc0 = fmaf(qb.x, __uint_as_float(kw.z << 16), sc0);
-            sc1 = fmaf(qb.y, __uint_as_float(kw.z & 0xffff0000u), sc1);
-            sc0 = fmaf(qb.z, __uint_as_float(kw.w << 16), sc0);
-            sc1 = fmaf(qb.w, __uint_as_float(kw.w & 0xffff0000u), sc1);
-        }
-        const float sc = (r < valid) ? (sc0 + sc1) * a.scale_log2 : -INFINITY;   // log2 domain
-        float mx = sc;
+        for (int kk = 0; kk < D / 16; ++kk) {
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-        if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = mx;
-        __syncthreads();
-        const float m_new = fmaxf(m_run, fmaxf(sRed[h][0], sRed[h][1]));   // finite: key 0 of every page is valid
-        const float alpha = exp2f(m_run - m_new);                           // 0 on the first page
-        const float p = exp2f(sc - m_new);
-        sP[h][r] = p;
-        float sum = p;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        __syncthreads();                                 // sRed reads done, sP written
-        if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = sum;
-        __syncthreads();
-        l_run = l_run * alpha + (sRed[h][0] + sRed[h][1]);
-        m_run = m_new;
-        acc[0] *= alpha;
-        acc[1] *= alpha;
-        if (kColsPerThread == 2) {
-            for (int k4 = 0; k4 < valid; k4 += 4) {      // never touch V rows past the newest token
-                const float4 pk = *reinterpret_cast<const float4*>(&sP[h][k4]);
-                const float pv[4] = {pk.x, pk.y, pk.z, pk.w};
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    if (k4 + q4 < valid) {
-                        const uint32_t vw = sV[k4 + q4][r];
-                        acc[0] = fmaf(pv[q4], __uint_as_float(vw << 16), acc[0]);
-                        acc[1] = fmaf(pv[q4], __uint_as_float(vw & 0xffff0000u), acc[1]);
-                    }
-                }
+            for (int nt = 0; nt < 2; ++nt) {
+                const int key = key0 + nt * 8 + gid;     // B fragment: n = gid, k = 2*tig (+8)
+                const uint32_t row = kb + key * kRowBytes + tig * 4;
+                uint32_t b0, b1;
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(b0) : "r"(row + (((2 * kk) ^ (key & 7)) << 4)));
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(b1) : "r"(row + (((2 * kk + 1) ^ (key & 7)) << 4)));
+                mma_16816(sc[nt], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
             }
-        } else {
-            const __nv_bfloat16* sVh = reinterpret_cast<const __nv_bfloat16*>(&sV[0][0]);
-#pragma unroll 8
-            for (int k = 0; k < valid; ++k) acc[0] = fmaf(sP[h][k], __bfloat162float(sVh[k * D + c0]), acc[0]);
         }
-        __syncthreads();                                 // sP, sRed and this stage are free again
+        // lane (gid < 2, tig) holds head gid's scores of keys key0 + nt*8 + 2*tig, +1
+        float sv[4];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int key = key0 + (i >> 1) * 8 + 2 * tig + (i & 1);
+            sv[i] = (gid < 2) ? ((key < valid) ? sc[i >> 1][i & 1] * a.scale_log2 : -INFINITY) : 0.f;
+            mx = fmaxf(mx, sv[i]);
+        }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));       // finite: key0 < valid
+        const float m_new = fmaxf(m_run, mx);
+        const float alpha = exp2f(m_run - m_new);                   // 0 on the warp's first page
+        float pv[4], psum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            pv[i] = exp2f(sv[i] - m_new);
+            psum += pv[i];
+        }
+        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+        l_run = l_run * alpha + psum;
+        m_run = m_new;
+        // P as the A operand of the second mma: the C layout of the scores is the A layout of the next k-step
+        const uint32_t pa0 = gid < 2 ? pack_bf16x2(pv[0], pv[1]) : 0u;   // keys 2*tig, +1
+        const uint32_t pa2 = gid < 2 ? pack_bf16x2(pv[2], pv[3]) : 0u;   // keys 8 + 2*tig, +1
+        // ---- O = alpha * O + P V: D / 8 n-tiles of 8 columns, V fragments by ldmatrix.trans ---------
+        const int lrow = key0 + (lane & 7) + ((lane >> 3) & 1) * 8;      // ldmatrix: lane supplies row (lane % 8) of matrix lane / 8
+        const uint32_t vrow = vb + lrow * kRowBytes;
+#pragma unroll
+        for (int dn = 0; dn < D / 8; dn += 2) {
+            acc[dn][0] *= alpha;
+            acc[dn][1] *= alpha;
+            acc[dn + 1][0] *= alpha;
+            acc[dn + 1][1] *= alpha;
+            uint32_t r0, r1, r2, r3;   // matrices: (keys 0-7, dn), (keys 8-15, dn), (keys 0-7, dn+1), (keys 8-15, dn+1)
+            ldmatrix_x4_trans(vrow + (((dn + (lane >> 4)) ^ (lrow & 7)) << 4), r0, r1, r2, r3);
+            mma_16816(acc[dn], pa0, 0u, pa2, 0u, r0, r1);
+            mma_16816(acc[dn + 1], pa0, 0u, pa2, 0u, r2, r3);
+        }
     }
-    const float inv = 1.f / l_run;
+    cp_async_wait<0>();
+    // ---- merge the four warps' states ------------------------------------------------------------------
+    if (gid < 2) {
+        if (tig == 0) { sM[warp][gid] = m_run; sL[warp][gid] = l_run; }
+#pragma unroll
+        for (int dn = 0; dn < D / 8; ++dn) {
+            sO[warp][gid][dn * 8 + 2 * tig] = acc[dn][0];
+            sO[warp][gid][dn * 8 + 2 * tig + 1] = acc[dn][1];
+        }
+    }
+    __syncthreads();
+    const int h = tid >> 6, r = tid & 63;
+    float m_all = fmaxf(fmaxf(sM[0][h], sM[1][h]), fmaxf(sM[2][h], sM[3][h]));   // warp 0 always has key 0
+    float wgt[4], l_all = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        wgt[w] = exp2f(sM[w][h] - m_all);                // 0 for a warp that never saw a valid key
+        l_all = fmaf(wgt[w], sL[w][h], l_all);
+    }
+    const float inv = 1.f / l_all;
+    constexpr int kColsPerThread = D / 64;
     __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + kvh * 2 + h) * D;
 #pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c) orow[c0 + c] = __float2bfloat16_rn(acc[c] * inv);
-    if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    for (int c = 0; c < kColsPerThread; ++c) {
+        const int col = r * kColsPerThread + c;
+        float o = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) o = fmaf(wgt[w], sO[w][h][col], o);
+        orow[col] = __float2bfloat16_rn(o * inv);
+    }
+    if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
 // One thread per sequence: Eq. 1 for the block of the newest token, mapped through the page table.
@@ -460,7 +521,10 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
         BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 64 * 2));
         BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     }
-    if ((int64_t)batch * hkv >= sm_count[dev]) {
+#ifndef BF1_DEC_FUSED_DIV
+#define BF1_DEC_FUSED_DIV 1
+#endif
+    if ((int64_t)batch * hkv * BF1_DEC_FUSED_DIV >= sm_count[dev]) {
         // enough (sequence, KV head) pairs to fill the GPU: one CTA walks a whole list
         dim3 grid(hkv, batch);
         if (d == 128) decode_fused_kernel<128><<<grid, kDecThreads, kDecStages * 2 * 64 * 128 * 2, (cudaStream_t)stream>>>(a);
