@@ -193,9 +193,60 @@ def time_region(fn, reps, stream):
     return statistics.median(out)
 
 
-def sweep(bf1, dev):
-    """BF1 vs the library's dense-causal mode, per layer, with the paper's protocol (Section
-    4.3): 5 warm-ups, 30 repetitions, two opposite pattern orders, median of the order medians."""
+GRAPH_LAUNCHES = 16
+
+
+def graph_timer(fn, dev, launches=GRAPH_LAUNCHES):
+    """Capture `launches` back-to-back calls of fn() in a CUDA graph on a side stream and return
+    replay(reps) -> list of per-launch times in ms (CUDA events around each replay).  The GPU runs
+    the launches without the host in between, so the figure is kernel time: launch gaps of a busy
+    stream included, Python, ctypes and driver latency of an idle one excluded."""
+    side = torch.cuda.Stream(device=dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            fn()
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(launches):
+                fn()
+
+    def replay(reps):
+        out = []
+        with torch.cuda.stream(side):
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(side)
+                graph.replay()
+                e1.record(side)
+                e1.synchronize()
+                out.append(e0.elapsed_time(e1) / launches)
+        return out
+    return replay
+
+
+def timed_with_clock(replay, local_rank, reps=30, min_ms=40.0):
+    """Median per-launch time of `reps` replays, then the median SM clock sampled (read-only NVML) while
+    the same graph keeps replaying for at least `min_ms`: (ms, MHz or None)."""
+    ts = replay(reps)
+    ms = statistics.median(ts)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t0 = time.perf_counter()
+    while (time.perf_counter() - t0) * 1e3 < min_ms:
+        replay(4)
+    clk = sampler.stop()
+    return ms, clk["sm_mhz"]
+
+
+def sweep(bf1, dev, local_rank=0):
+    """BF1 vs the library's dense-causal mode, per layer, with the paper's protocol (Section 4.3):
+    5 warm-ups, 30 repetitions, two opposite pattern orders, median of the order medians.  A repetition
+    is one replay of a CUDA graph of 16 launches (kernel-only time per launch); `*_host_inclusive_ms` is
+    the same protocol with one Python call between two events on an idle stream, i.e. what a caller
+    that launches a single layer and waits would see.  Each point also carries the median SM clock
+    while it ran and time x clock (kilo-cycles), so that a point measured while the clocks were
+    still pulled down by a long dense launch can be told from a slow kernel."""
     out = []
     for name in ("qwen_2k", "qwen_4k", "qwen_8k", "qwen_16k", "qwen_32k"):
         w = I.WORKLOADS[name]
@@ -208,24 +259,44 @@ def sweep(bf1, dev):
         f_s = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
         work = torch.zeros(4, dtype=torch.int32, device=dev)
         f_d = lambda: bf1.dense_causal_fwd(q, k, v, cu, w.max_seqlen, out=o, lse=lse, work=work)
+        torch.cuda.synchronize()
+        g_s, g_d = graph_timer(f_s, dev), graph_timer(f_d, dev)
         meds = {"bf1": [], "dense": []}
+        host = {"bf1": [], "dense": []}
+        mhz = {"bf1": [], "dense": []}
         for order in (("dense", "bf1"), ("bf1", "dense")):
             for which in order:
+                g = g_s if which == "bf1" else g_d
+                g(5)
+                ms, clk = timed_with_clock(g, local_rank)
+                meds[which].append(ms)
+                if clk:
+                    mhz[which].append(clk)
                 f = f_s if which == "bf1" else f_d
                 for _ in range(5):
                     f()
-                meds[which].append(time_region(f, 30, stream))
+                host[which].append(time_region(f, 30, stream))
         ms_s, ms_d = statistics.median(meds["bf1"]), statistics.median(meds["dense"])
         n = w.seqlens[0]
         pairs = selected_pairs(n)
         m = int(math.log2(n // 64))
         closed = n * 64 * m - 64 * 64 * m + n * 65 // 2        # n log n total for n = 64 * 2^m (Prop. 1's accounting)
-        out.append({"n": n, "bf1_ms": round(ms_s, 5), "dense_ms": round(ms_d, 5), "speedup": round(ms_d / ms_s, 3),
-                    "bf1_tflops": round(flops(pairs, w.d, w.hq) / ms_s / 1e9, 1),
-                    "dense_tflops": round(flops(n * (n + 1) // 2, w.d, w.hq) / ms_d / 1e9, 1),
-                    "selected_pairs_planner": int(route.total_pairs.item()), "selected_pairs_closed_form": closed,
-                    "pair_reduction": round(n * (n + 1) / 2 / pairs, 3), "inputs": "L2-warm (same buffers re-run)"})
-        del q, k, v, o, lse
+        point = {"n": n, "bf1_ms": round(ms_s, 5), "dense_ms": round(ms_d, 5), "speedup": round(ms_d / ms_s, 3),
+                 "bf1_tflops": round(flops(pairs, w.d, w.hq) / ms_s / 1e9, 1),
+                 "bf1_frac_of_bf16_peak": round(flops(pairs, w.d, w.hq) / ms_s / 1e9 / measured_peaks()["bf16_tflops"], 4),
+                 "dense_tflops": round(flops(n * (n + 1) // 2, w.d, w.hq) / ms_d / 1e9, 1),
+                 "bf1_host_inclusive_ms": round(statistics.median(host["bf1"]), 5),
+                 "dense_host_inclusive_ms": round(statistics.median(host["dense"]), 5),
+                 "selected_pairs_planner": int(route.total_pairs.item()), "selected_pairs_closed_form": closed,
+                 "pair_reduction": round(n * (n + 1) / 2 / pairs, 3),
+                 "timing": "CUDA graph of %d launches per repetition" % GRAPH_LAUNCHES,
+                 "inputs": "L2-warm (same buffers re-run)"}
+        if mhz["bf1"] and mhz["dense"]:
+            c_s, c_d = statistics.median(mhz["bf1"]), statistics.median(mhz["dense"])
+            point.update({"bf1_sm_mhz": c_s, "dense_sm_mhz": c_d, "bf1_kcycles": round(ms_s * c_s, 1),
+                          "dense_kcycles": round(ms_d * c_d, 1), "speedup_in_cycles": round(ms_d * c_d / (ms_s * c_s), 3)})
+        out.append(point)
+        del q, k, v, o, lse, g_s, g_d
     # the ragged batch (3001, 8192, 12345, 16384 tokens) in one varlen launch
     w = I.WORKLOADS["ragged"]
     q, k, v = (t.to(dev) for t in I.draw_qkv(w))
@@ -234,9 +305,10 @@ def sweep(bf1, dev):
     o = torch.empty_like(q)
     lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
     f = lambda: bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
-    for _ in range(5):
-        f()
-    ms = time_region(f, 30, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    g = graph_timer(f, dev)
+    g(5)
+    ms = statistics.median(g(30))
     pairs = sum(selected_pairs(x) for x in w.seqlens)
     out.append({"ragged_seqlens": list(w.seqlens), "bf1_ms": round(ms, 5),
                 "bf1_tflops": round(flops(pairs, w.d, w.hq) / ms / 1e9, 1),
@@ -244,33 +316,52 @@ def sweep(bf1, dev):
     return out
 
 
+def host_route_arrays(lists, n, block=64):
+    """Arrays for bf1.Route.from_host from explicit per-block lists of one sequence of n tokens."""
+    counts = [len(x) for x in lists]
+    deg = max(counts)
+    kv_idx = [list(x) + [-1] * (deg - len(x)) for x in lists]
+    pairs = []
+    for j, x in enumerate(lists):
+        rows = min(block, n - j * block)
+        pairs.append(rows * block * (len(x) - 1) + rows * (rows + 1) // 2)
+    order = sorted(range(len(lists)), key=lambda g: (-counts[g], g))
+    return dict(qb_seq=[0] * len(lists), qb_block=list(range(len(lists))), kv_count=counts, kv_idx=kv_idx,
+                pair_count=pairs, order=order, total_pairs=sum(pairs))
+
+
 def topology_sweep(bf1, dev):
     """Does the route's topology change the kernel's cost?  (Section 5.1: equal-pair-count BF1, sliding and
     static-random routes have nearly identical sparse kernel time.)  One 32K layer through routes with about
-    the same number of block pairs: BF1, a sliding window with the closest pair count, BF1 without block 0,
-    dyadic predecessors without a local window.  Reported per executed tile so that small differences in
-    the pair budget cancel."""
+    the same number of block pairs: BF1, a sliding window with the closest pair count, a seeded static-random
+    non-local graph with exactly BF1's list lengths (uploaded from the host, not planned), BF1 without block
+    0, dyadic predecessors without a local window.  Kernel time from a CUDA graph of 16 launches; reported
+    per executed tile as well, so that small differences in the pair budget cancel."""
     w = I.WORKLOADS["qwen_32k"]
     n = w.seqlens[0]
     q, k, v = (t.to(dev) for t in I.draw_qkv(w))
     cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
     o = torch.empty_like(q)
     lse = torch.empty((w.hq, w.total_tokens), dtype=torch.float32, device=dev)
-    stream = torch.cuda.current_stream()
     nb = n // 64
     target = sum(degree(j) for j in range(nb))
     best_w = min(range(1, 64), key=lambda ww: abs(sum(min(j, ww) + 1 for j in range(nb)) - target))
     routes = [("bf1", bf1.RouteCfg()), ("sliding W=%d (equal block-pair budget)" % best_w,
                                         bf1.RouteCfg(local_blocks=best_w, global_first=0, dyadic=0)),
+              ("static random graph (seed 17, BF1's list lengths, host-built lists)", None),
               ("bf1 without block 0", bf1.RouteCfg(global_first=0)),
               ("dyadic only (W=0)", bf1.RouteCfg(local_blocks=0, global_first=0, dyadic=1))]
     out = []
     for name, cfg in routes:
-        route = bf1.plan_route(cu, n, cfg)
+        if cfg is None:
+            route = bf1.Route.from_host(device=dev, **host_route_arrays(I.static_random_lists(nb, seed=17), n))
+        else:
+            route = bf1.plan_route(cu, n, cfg)
         f = lambda: bf1.attn_fwd(q, k, v, cu, n, route, out=o, lse=lse)
-        for _ in range(5):
-            f()
-        ms = time_region(f, 30, stream)
+        torch.cuda.synchronize()
+        g = graph_timer(f, dev)
+        g(5)
+        ms = statistics.median(g(30))
         route.check_status()
         tiles = int(route.kv_count[:nb].sum().item()) * w.hkv
         out.append({"route": name, "block_pairs": tiles // w.hkv, "ms": round(ms, 5),
@@ -594,7 +685,7 @@ def run_ours(args):
                      "kernel_ms_per_launch": kern_ms},
     }
     if not args.no_sweep and world == 1:
-        line["sweep"] = sweep(bf1, dev)
+        line["sweep"] = sweep(bf1, dev, local_rank)
         line["decode"] = decode_sweep(bf1, dev)
         line["backward"] = backward_sweep(bf1, dev)
         line["topology"] = topology_sweep(bf1, dev)
@@ -625,6 +716,19 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def spawn_ranks(n: int) -> int:
+    """`bench.py --gpus N` started bare: run this same command line as N ranks (one process per GPU)
+    under torch.distributed.run on this node and pass its exit code on."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd).returncode
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -637,6 +741,8 @@ def main():
                     help="only time `--steps` launches of one workload (used for profiling)")
     ap.add_argument("--mode", default="bf1", choices=["bf1", "dense", "decode", "bwd"])
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.single:
+        sys.exit(spawn_ranks(args.gpus))
     if args.single:
         run_single(args)
     elif args.impl == "reference":

@@ -98,16 +98,39 @@ def draw_qkv(w: Workload, layer: int = 0):
     return q.to(torch.bfloat16), k.to(torch.bfloat16), v.to(torch.bfloat16)
 
 
-def mutate_after(w: Workload, q, k, v, seq: int, t: int, seed: int):
+def static_random_lists(num_blocks: int, seed: int, local_blocks: int = 2):
+    """A fixed random non-local block graph with the BF1 route's per-block list lengths: for query
+    block j the list is j itself plus a seeded random subset of its predecessors, as many as the
+    paper's route reads for that block (Section 4.3's static-random control; the paper does not give
+    its construction, so this one is this repository's own).  Returns one ascending list per block,
+    self block last.  Pure index bookkeeping: no attention arithmetic."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(int(seed))
+    lists = []
+    for j in range(num_blocks):
+        want = {j, 0} | {j - w for w in range(1, local_blocks + 1) if j - w >= 0}
+        k = 0
+        while j - (1 << k) >= 0:
+            want.add(j - (1 << k))
+            k += 1
+        npred = len(want) - 1                      # predecessors the paper's route reads for block j
+        perm = torch.randperm(j, generator=g)[:npred].tolist() if j > 0 else []
+        lists.append(sorted(perm) + [j])
+    return lists
+
+
+def mutate_after(w: Workload, q, k, v, seq: int, t: int, seed: int, gain: float = 1.0):
     """Copies of (q, k, v) in which every token of sequence ``seq`` at position > t is
-    replaced by fresh finite N(0,1) values (the future-token mutation gate, Section 4.2)."""
+    replaced by fresh finite N(0,1) values (the future-token mutation gate, Section 4.2).
+    ``gain`` scales the new Q and K rows: large values make the scores of the mutated rows jump
+    from tile to tile by far more than those of the rows that must stay untouched."""
     g = torch.Generator(device="cpu")
     g.manual_seed(int(seed))
     cu = w.cu_seqlens()
     lo, hi = cu[seq] + t + 1, cu[seq + 1]
     q2, k2, v2 = q.clone(), k.clone(), v.clone()
     if hi > lo:
-        q2[lo:hi] = torch.randn((hi - lo, w.hq, w.d), generator=g).to(torch.bfloat16)
-        k2[lo:hi] = torch.randn((hi - lo, w.hkv, w.d), generator=g).to(torch.bfloat16)
+        q2[lo:hi] = (gain * torch.randn((hi - lo, w.hq, w.d), generator=g)).to(torch.bfloat16)
+        k2[lo:hi] = (gain * torch.randn((hi - lo, w.hkv, w.d), generator=g)).to(torch.bfloat16)
         v2[lo:hi] = torch.randn((hi - lo, w.hkv, w.d), generator=g).to(torch.bfloat16)
     return q2, k2, v2

@@ -98,8 +98,9 @@ typedef struct {
 } bf1_route;
 
 /* Host-only helper: how large the route arrays must be for a batch of `batch` sequences,
- * `total_tokens` tokens in all, none longer than `max_seqlen`.  capacity_qblocks is an
- * upper bound on sum_s ceil(n_s / b); max_degree is the largest |P(j)| any block of a
+ * `total_tokens` tokens in all, none longer than `max_seqlen`.  capacity_qblocks is the
+ * largest value sum_s ceil(n_s / b) can take for that batch size and token total (exact for
+ * batch = 1); max_degree is the largest |P(j)| any block of a
  * sequence of max_seqlen tokens has (Proposition 1).  Touches no device. */
 int bf1_route_capacity(int32_t batch, int64_t total_tokens, int32_t max_seqlen,
                        const bf1_route_cfg *cfg /* host */,
@@ -154,10 +155,14 @@ int bf1_dense_causal_fwd(const void *q, const void *k, const void *v,
  *   status_dev  optional [1] int32 device word that receives the BF1_DEV_* bits (written by the
  *               planner, OR-ed by the attention kernel); NULL keeps them inside the library
  *   other arguments as bf1_attn_fwd
- * Limits: the batch may hold at most 4096 query blocks (sum of ceil(n_s / 64); 262,144 tokens
- * for lengths that are multiples of 64) and lists of at most 32 entries (the paper's route
- * needs 3 + floor(log2(B-1))).  Beyond that the call returns BF1_ERR_CAPACITY and launches
- * nothing.  It calls no cudaMalloc / cudaFree / allocating library routine.  The first call on a
+ * Limits: the batch may hold at most 4096 query blocks and lists of at most 32 entries (the
+ * paper's route needs 3 + floor(log2(B-1))).  The block count is checked on the host through
+ * bf1_route_capacity's upper bound for (batch, total_tokens): one sequence of 262,144 tokens
+ * (exactly 4096 blocks) is accepted, a batch of B sequences may hold 64 * (4096 - B) + B tokens.
+ * Beyond that the call returns BF1_ERR_CAPACITY and launches nothing; so do host-checkable
+ * argument errors, before the planner runs.  With status_dev == NULL a device-side refusal
+ * (BF1_DEV_BAD_SEQLENS from the planner, which then leaves o and lse unwritten) cannot be read
+ * back by the caller: pass a status word when the lengths are not trusted.  It calls no cudaMalloc / cudaFree / allocating library routine.  The first call on a
  * device looks up the array's address; make it before any stream capture.  All calls share the
  * array and overwrite the previous call's contents, so calls that may overlap on the GPU
  * (streams without ordering between them) race and must be avoided. */
@@ -172,8 +177,8 @@ int bf1_attn_fwd_noalloc(const void *q, const void *k, const void *v, const int3
  * the pages of P(j), the self page only up to token n-1: O(log B) pages per step.  The KV cache is
  * paged: k_pages / v_pages are [num_pages, 64, hkv, d] bf16 and page_table[s, i] names the
  * physical page that holds logical block i of sequence s.  The page list changes only when n
- * crosses a block boundary, so one plan serves a whole 64-token route epoch (the paper's open
- * item: "persistent plan reuse across a 64-token route epoch"). */
+ * crosses a block boundary, so one plan serves a whole 64-token route epoch (Section 5.4 names
+ * keeping a plan alive across such an epoch as the open systems problem). */
 typedef struct {
     int32_t  max_degree;   /* host: row pitch of `page`                                          */
     int32_t *count;        /* [batch] pages to read for the sequence (0 for an empty sequence)   */
@@ -210,8 +215,8 @@ int bf1_decode_fwd(const void *q, const void *k_pages, const void *v_pages, int3
                    float softmax_scale, const bf1_decode_plan *plan /* host */, void *workspace,
                    void *o, float *lse, void *stream);
 
-/* ---- backward over the same route (Section 4.2 gates on "forward and backward with finite Q/K/V
- * gradients") -------------------------------------------------------------------------------------
+/* ---- backward over the same route (Section 4.2's gates include a backward pass with finite
+ * Q, K and V gradients) ---------------------------------------------------------------------------
  * Given the forward's inputs, its outputs o and lse, and the upstream gradient d_o [T, hq, d] bf16,
  * writes dq [T, hq, d], dk and dv [T, hkv, d] in bf16 (the gradients of the G query heads of a KV
  * head add up in dk, dv).  P is recomputed as exp(scale * <q, k> - lse); dk and dv are accumulated

@@ -149,6 +149,22 @@ class Route:
                       r.sched.data_ptr())
         return r
 
+    @staticmethod
+    def from_host(qb_seq, qb_block, kv_count, kv_idx, pair_count, order, total_pairs: int, device,
+                  cfg: Optional[RouteCfg] = None) -> "Route":
+        """Upload a route the caller built on the host (any ascending lists whose last entry is the
+        query block itself; kv_idx [slots, max_degree] padded with -1).  Marshalling only."""
+        kv_idx = torch.as_tensor(kv_idx, dtype=torch.int32)
+        slots, max_degree = kv_idx.shape
+        r = Route.empty(max(slots, 1), max_degree, device, cfg)
+        for name, src in (("qb_seq", qb_seq), ("qb_block", qb_block), ("kv_count", kv_count),
+                          ("pair_count", pair_count), ("order", order)):
+            getattr(r, name)[:slots].copy_(torch.as_tensor(src, dtype=torch.int32))
+        r.kv_idx[:slots].copy_(kv_idx)
+        r.total_pairs.fill_(int(total_pairs))
+        r.num_qblocks.fill_(slots)
+        return r
+
     def check_status(self):
         """Synchronising read of the device status word; raises if any BF1_DEV_* bit is set."""
         st = int(self.status.item())

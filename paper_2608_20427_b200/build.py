@@ -29,9 +29,7 @@ def is_stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False, out: str = None, defines=()) -> str:
     """Compile the library if it is missing or older than its sources; return its path.
-    `out` / `defines` build a variant (e.g. -DBF1_TRACE) somewhere else."""
-    if out is None and os.environ.get("BF1_LIB"):
-        return os.environ["BF1_LIB"]          # use a library built elsewhere (e.g. a trace build)
+    `out` / `defines` compile a variant of the sources to another path (the binding never loads it)."""
     if out is None and not force and not is_stale():
         return LIB
     lib = out or LIB

@@ -1,6 +1,6 @@
 // BF1 attention backward (dQ, dK, dV) over the same route, for sm_100a, head dimension 128.
 //
-// The paper gates its operator on "forward and backward with finite Q/K/V gradients" (Section
+// The paper's correctness gates include a backward pass with finite Q, K and V gradients (Section
 // 4.2).  With P = exp(S - LSE) recomputed from the saved LSE and D_i = <dO_i, O_i>:
 //     dV_p += P^T dO,   dP = dO V_p^T,   dS = P o (dP - D) * scale,   dQ += dS K_p,   dK_p += dS^T Q.
 // Work unit = (query block, KV head) as in the forward pass: the two grouped query heads are the

@@ -403,8 +403,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
 // One thread per sequence: Eq. 1 for the block of the newest token, mapped through the page table.
 __global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_table, int max_pages_per_seq,
                                    int batch, bf1_route_cfg cfg, bf1_decode_plan plan) {
+    // the status word is cleared by a memset in front of this launch, so every thread may OR into it
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s == 0) *plan.status = 0;
     if (s >= batch) return;
     const int n = seqlens[s];
     int32_t* list = plan.page + (size_t)s * plan.max_degree;
@@ -468,6 +468,7 @@ extern "C" int bf1_plan_decode(const int32_t* seqlens_dev, const int32_t* page_t
         return fail(BF1_ERR_CAPACITY, "decode plan max_degree %d < %d needed for %d pages per sequence", out->max_degree,
                     need, max_pages_per_seq);
     if (batch == 0) return BF1_OK;
+    BF1_CUDA_CHECK(cudaMemsetAsync(out->status, 0, sizeof(int32_t), (cudaStream_t)stream));
     plan_decode_kernel<<<(batch + 127) / 128, 128, 0, (cudaStream_t)stream>>>(seqlens_dev, page_table_dev,
                                                                                max_pages_per_seq, batch, *cfg, *out);
     BF1_CUDA_CHECK(cudaGetLastError());
@@ -521,10 +522,7 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
         BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 64 * 2));
         BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     }
-#ifndef BF1_DEC_FUSED_DIV
-#define BF1_DEC_FUSED_DIV 1
-#endif
-    if ((int64_t)batch * hkv * BF1_DEC_FUSED_DIV >= sm_count[dev]) {
+    if ((int64_t)batch * hkv >= sm_count[dev]) {
         // enough (sequence, KV head) pairs to fill the GPU: one CTA walks a whole list
         dim3 grid(hkv, batch);
         if (d == 128) decode_fused_kernel<128><<<grid, kDecThreads, kDecStages * 2 * 64 * 128 * 2, (cudaStream_t)stream>>>(a);

@@ -10,9 +10,13 @@
 // What to know:
 //   - The array is kScratchBytes (about 0.6 MB) of device memory on every GPU that loads the
 //     library, held until the process exits.
-//   - Limits: at most kMaxQBlocks query blocks in the batch (sum over sequences of
-//     ceil(n / 64); 4096 blocks = 262,144 tokens when lengths are multiples of 64) and lists of
-//     at most kMaxDegree entries.  Larger requests return BF1_ERR_CAPACITY and launch nothing.
+//   - Limits: at most kMaxQBlocks query blocks in the batch and lists of at most kMaxDegree
+//     entries.  The host does not know the individual lengths, so the block count it checks is
+//     bf1_route_capacity's upper bound for (batch, total_tokens): one sequence of 262,144 tokens
+//     is exactly 4096 blocks and is accepted; a batch of B sequences may hold
+//     64 * (4096 - B) + B tokens.  Larger requests return BF1_ERR_CAPACITY and launch nothing.
+//   - Host-checkable argument errors (null or misaligned pointers, unsupported geometry) are
+//     reported before the planner is launched.
 //   - The first call on a device looks up the array's device address (no allocation); make
 //     that first call outside any stream capture.
 //   - Every call uses the same array and overwrites what the previous call left (the planner
@@ -20,6 +24,12 @@
 //     Calls that can overlap on the GPU -- different streams without ordering -- race on it.
 //   - No cudaMalloc, cudaFree or allocating library routine is called.
 #include "bf1_common.cuh"
+
+namespace bf1 {
+int check_attn_args(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_dev, int32_t batch,
+                    int64_t total_tokens, int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d, const void* o,
+                    const float* lse);   // bf1_attn.cu
+}
 
 namespace {
 
@@ -69,6 +79,8 @@ extern "C" int bf1_attn_fwd_noalloc(const void* q, const void* k, const void* v,
                                     int32_t batch, int64_t total_tokens, int32_t max_seqlen, int32_t hq,
                                     int32_t hkv, int32_t d, float softmax_scale, const bf1_route_cfg* cfg,
                                     void* o, float* lse, int32_t* status_dev, void* stream) {
+    if (int rc = bf1::check_attn_args(q, k, v, cu_seqlens_dev, batch, total_tokens, max_seqlen, hq, hkv, d, o, lse))
+        return rc;
     int32_t need_blocks = 0, need_degree = 0;
     if (int rc = bf1_route_capacity(batch, total_tokens, max_seqlen, cfg, &need_blocks, &need_degree)) return rc;
     if (need_blocks > kMaxQBlocks)

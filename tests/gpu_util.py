@@ -71,3 +71,39 @@ def assert_parity(o_gpu, lse_gpu, o_ref, lse_ref, rows=None):
     assert e["o_rel_rms"] <= O_REL_RMS, e
     assert e["lse_max_abs"] <= LSE_ABS, e
     return e
+
+
+def host_route(lists_per_seq, seqlens, max_degree=None, block=64):
+    """Route arrays for `bf1.Route.from_host`, written by hand on the host from explicit lists
+    (one list of ascending KV block indices per query block, self block last): slots numbered
+    sequence by sequence, pair counts by Proposition 1's accounting, hand-out order by
+    descending list length.  Returns (arrays dict, total_pairs)."""
+    qb_seq, qb_block, counts, pairs, rows_idx = [], [], [], [], []
+    for s, (lists, n) in enumerate(zip(lists_per_seq, seqlens)):
+        assert len(lists) == (n + block - 1) // block
+        for j, lst in enumerate(lists):
+            assert lst == sorted(set(lst)) and lst[-1] == j and lst[0] >= 0
+            rows = min(block, n - j * block)
+            qb_seq.append(s)
+            qb_block.append(j)
+            counts.append(len(lst))
+            pairs.append(rows * block * (len(lst) - 1) + rows * (rows + 1) // 2)
+            rows_idx.append(lst)
+    deg = max_degree or max(counts)
+    kv_idx = np.full((len(counts), deg), -1, dtype=np.int32)
+    for g, lst in enumerate(rows_idx):
+        kv_idx[g, :len(lst)] = lst
+    order = sorted(range(len(counts)), key=lambda g: (-counts[g], g))
+    arrays = dict(qb_seq=qb_seq, qb_block=qb_block, kv_count=counts, kv_idx=kv_idx, pair_count=pairs, order=order)
+    return arrays, int(sum(pairs))
+
+
+def mask_from_lists(lists, n, block=64):
+    """n x n boolean token mask of one sequence: listed blocks in full, the self block causally."""
+    m = np.zeros((n, n), dtype=bool)
+    for j, lst in enumerate(lists):
+        r0, r1 = j * block, min((j + 1) * block, n)
+        for p in lst:
+            c0, c1 = p * block, min((p + 1) * block, n)
+            m[r0:r1, c0:c1] = True
+    return m & np.tril(np.ones((n, n), dtype=bool))

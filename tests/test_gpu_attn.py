@@ -92,6 +92,32 @@ def test_future_token_isolation_is_bitwise():
         assert not np.array_equal(o[t + 1:], o2[t + 1:])
 
 
+@pytest.mark.parametrize("dense", [False, True], ids=["bf1", "dense"])
+@pytest.mark.parametrize("hq,hkv", [(4, 2), (8, 2)], ids=["G2", "G4"])
+def test_future_token_isolation_is_bitwise_when_later_rows_rescale(dense, hq, hkv):
+    """The same gate on the path where it could fail: the kernel rescales a row's accumulator only
+    when that row's maximum jumps by more than 2^8 between tiles, and the rows of one warp are
+    consecutive tokens.  The mutated tokens get Q and K rows 36x larger, so that they jump in nearly
+    every tile while the untouched rows never do; t sits in the middle of a 32-row group, so untouched
+    and mutated rows share a warp.  Rows up to t must not change in a single bit."""
+    n = 600
+    w = I.custom([n], hq=hq, hkv=hkv, d=128, seed=650 + hq)
+    q, k, v = I.draw_qkv(w)
+    o, lse, _ = run_gpu(w, q, k, v, dense=dense)
+    for t in (305, 337 + 12, 46):          # positions 17, 29 and 14 of their 32-row groups
+        q2, k2, v2 = I.mutate_after(w, q, k, v, 0, t, seed=750 + t, gain=36.0)
+        o2, lse2, _ = run_gpu(w, q2, k2, v2, dense=dense)
+        assert np.array_equal(o[:t + 1], o2[:t + 1]) and np.array_equal(lse[:, :t + 1], lse2[:, :t + 1])
+        # the mutation did reach the later rows, and by the amounts the oracle predicts: their
+        # scores are ~1300 times larger, so LSE moves by hundreds
+        rows = np.arange(t + 1, n)
+        o_ref, lse_ref = oracle_full(w, q2, k2, v2, dense=dense, rows=rows)
+        assert np.abs(lse_ref[:, rows] - lse[:, rows]).min() > 50.0
+        assert np.abs(lse2[:, rows] - lse_ref[:, rows]).max() <= 1e-3 * np.abs(lse_ref[:, rows]).max()
+        diff = o2[rows].astype(np.float64) - o_ref[rows]
+        assert np.sqrt((diff ** 2).mean() / (o_ref[rows].astype(np.float64) ** 2).mean()) <= 1e-2
+
+
 def test_zero_queries_give_log_count():
     """Q = 0: every selected key gets the same weight, so LSE = ln(#selected columns)."""
     n = 1000
@@ -137,3 +163,36 @@ def test_user_supplied_route_is_followed_and_bad_entries_are_flagged():
     bf1.attn_fwd(q.to(dev), k.to(dev), v.to(dev), cu, 1000, route)
     torch.cuda.synchronize()
     assert int(route.status.item()) & 8
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(4, 2, 128), (8, 2, 64)], ids=["G2-d128", "G4-d64"])
+def test_static_random_route_written_by_hand(hq, hkv, d):
+    """Section 4.3's static-random control: a route the planner did not write.  The test builds, on
+    the host, a seeded random non-local block graph with the BF1 route's list lengths for two
+    sequences (one with a partial last block), uploads it as a bf1_route and compares the kernel
+    with the oracle's defining form under the boolean mask made from the very same lists."""
+    from gpu_util import host_route, mask_from_lists
+    lens = [4096, 1000]
+    w = I.custom(lens, hq=hq, hkv=hkv, d=d, seed=1200 + d)
+    q, k, v = I.draw_qkv(w)
+    lists = [I.static_random_lists((n + 63) // 64, seed=17 + s) for s, n in enumerate(lens)]
+    # the graph is non-local: most entries are neither the window, block 0 nor a dyadic predecessor
+    bf1_sets = [set(np.flatnonzero(row)) for row in O.block_mask(O.cfg(), lens[0])]
+    assert sum(len(set(lst) - bf1_sets[j]) for j, lst in enumerate(lists[0])) > 200
+    arrays, total = host_route(lists, lens)
+    dev = torch.device("cuda:0")
+    route = bf1.Route.from_host(device=dev, total_pairs=total, **arrays)
+    cu = bf1.cu_seqlens_tensor(lens, dev)
+    T = w.total_tokens
+    out = torch.full((T + 64, hq, d), float("nan"), dtype=torch.bfloat16, device=dev)
+    lse = torch.full((hq, T), float("nan"), dtype=torch.float32, device=dev)
+    bf1.attn_fwd(q.to(dev), k.to(dev), v.to(dev), cu, max(lens), route, out=out[:T], lse=lse)
+    torch.cuda.synchronize()
+    route.check_status()
+    assert torch.isnan(out[T:].float()).all()
+    o_gpu, lse_gpu = out[:T].float().cpu().numpy(), lse.cpu().numpy()
+    cu_h = w.cu_seqlens()
+    for s, n in enumerate(lens):
+        sl = slice(cu_h[s], cu_h[s + 1])
+        o_ref, lse_ref = O.attn_mask(q[sl], k[sl], v[sl], mask_from_lists(lists[s], n))
+        assert_parity(o_gpu[sl], lse_gpu[:, sl], o_ref, lse_ref)

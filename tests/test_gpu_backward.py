@@ -15,6 +15,7 @@ from gpu_util import oracle_cfg, lib_cfg
 pytestmark = pytest.mark.gpu
 REL_RMS = 1e-2          # P, dS and the outputs are bf16 (2^-9 relative each); observed 2e-3 .. 5e-3
 REL_MAX = 2e-2          # of the gradient's largest magnitude; observed <= 6e-3
+ZERO_ABS = 1e-4         # where the exact gradient is zero: fp32 rounding of O(10) dot products, times P <= 1
 
 
 def run_case(w, seed):
@@ -35,8 +36,15 @@ def run_case(w, seed):
         got = got.float().cpu().numpy().astype(np.float64)
         assert np.isfinite(got).all(), name
         diff = got - ref
-        scale = max(float(np.abs(ref).max()), 1e-2)     # a one-key row has dq = dk = 0 exactly
-        rms_ref = max(float(np.sqrt((ref ** 2).mean())), 1e-2)
+        scale = float(np.abs(ref).max())
+        if scale < 1e-9:
+            # a gradient that is zero by definition (a token whose only key is itself has dq = dk = 0):
+            # the kernel's D = <dO, O> and dP = <dO, V> differ by fp32 rounding only, so what is left
+            # must be tiny in absolute terms -- no relative floor to hide behind
+            assert float(np.abs(got).max()) <= ZERO_ABS, (name, float(np.abs(got).max()))
+            out[name] = (0.0, 0.0)
+            continue
+        rms_ref = float(np.sqrt((ref ** 2).mean()))
         out[name] = (float(np.sqrt((diff ** 2).mean())) / rms_ref, float(np.abs(diff).max()) / scale)
     return out
 
@@ -55,6 +63,17 @@ def test_gradients_4k_qwen_geometry():
     w = I.custom([4096], hq=16, hkv=8, d=128, seed=6100, sink_scale=4.0)
     res = run_case(w, seed=2)
     print("4k", res)
+    for name, (rms, mx) in res.items():
+        assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
+
+
+@pytest.mark.parametrize("n", [8192, 32768])
+def test_gradients_at_the_benchmarked_lengths(n):
+    """The sizes bench.py's `backward` block times: several waves of units, lists of 9 to 11 entries,
+    up to eleven query blocks adding into one KV block.  All of dQ, dK, dV against the fp64 oracle."""
+    w = I.custom([n], hq=16, hkv=8, d=128, seed=6200 + n)
+    res = run_case(w, seed=3)
+    print(n, res)
     for name, (rms, mx) in res.items():
         assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
 

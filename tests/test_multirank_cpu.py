@@ -62,3 +62,17 @@ def test_reference_arm_prints_one_line_from_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["gpu_launches"] == 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_bare_gpus_flag_spawns_its_own_ranks():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks itself (torch.distributed.run,
+    rendezvous on 127.0.0.1); the reference arm needs no GPU, so this runs here: one line, n_gpus 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR",
+                                                           "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [x for x in r.stdout.splitlines() if x.strip().startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
