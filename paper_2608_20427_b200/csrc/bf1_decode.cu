@@ -403,42 +403,48 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
 // One thread per sequence: Eq. 1 for the block of the newest token, mapped through the page table.
 __global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_table, int max_pages_per_seq,
                                    int batch, bf1_route_cfg cfg, bf1_decode_plan plan) {
-    // the status word is cleared by a memset in front of this launch, so every thread may OR into it
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= batch) return;
-    const int n = seqlens[s];
-    int32_t* list = plan.page + (size_t)s * plan.max_degree;
-    int deg = 0;
-    int bad = 0;
-    const int j = n > 0 ? (n - 1) / kPage : -1;
-    if (n < 0 || j >= max_pages_per_seq) bad = BF1_DEV_BAD_SEQLENS;
-    if (n > 0 && !bad) {
-        int last = -1, kmax = -1;
-        if (cfg.dyadic) while ((1 << (kmax + 1)) <= j) ++kmax;
-        int g = cfg.global_first ? 0 : 0x7fffffff;
-        int k = kmax;
-        int l = max(j - cfg.local_blocks, 0);
-        while (true) {                                   // merge of the three ascending candidate streams
-            const int dcur = (k >= 0) ? j - (1 << k) : 0x7fffffff;
-            const int lcur = (l <= j) ? l : 0x7fffffff;
-            const int m = min(g, min(dcur, lcur));
-            if (m == 0x7fffffff) break;
-            if (m == g) g = 0x7fffffff;
-            if (m == dcur) --k;
-            if (m == lcur) ++l;
-            if (m != last) {
-                if (deg < plan.max_degree) list[deg] = page_table[(size_t)s * max_pages_per_seq + m];
-                else bad |= BF1_DEV_CAPACITY;
-                ++deg;
-                last = m;
+    // One CTA walks the batch: error bits are collected in shared memory and the status word is
+    // WRITTEN once at the end, so no thread's bit can be lost to another thread's clearing store.
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    for (int s = threadIdx.x; s < batch; s += blockDim.x) {
+        const int n = seqlens[s];
+        int32_t* list = plan.page + (size_t)s * plan.max_degree;
+        int deg = 0;
+        int bad = 0;
+        const int j = n > 0 ? (n - 1) / kPage : -1;
+        if (n < 0 || j >= max_pages_per_seq) bad = BF1_DEV_BAD_SEQLENS;
+        if (n > 0 && !bad) {
+            int last = -1, kmax = -1;
+            if (cfg.dyadic) while ((1 << (kmax + 1)) <= j) ++kmax;
+            int g = cfg.global_first ? 0 : 0x7fffffff;
+            int k = kmax;
+            int l = max(j - cfg.local_blocks, 0);
+            while (true) {                                   // merge of the three ascending candidate streams
+                const int dcur = (k >= 0) ? j - (1 << k) : 0x7fffffff;
+                const int lcur = (l <= j) ? l : 0x7fffffff;
+                const int m = min(g, min(dcur, lcur));
+                if (m == 0x7fffffff) break;
+                if (m == g) g = 0x7fffffff;
+                if (m == dcur) --k;
+                if (m == lcur) ++l;
+                if (m != last) {
+                    if (deg < plan.max_degree) list[deg] = page_table[(size_t)s * max_pages_per_seq + m];
+                    else bad |= BF1_DEV_CAPACITY;
+                    ++deg;
+                    last = m;
+                }
             }
+            if (deg > plan.max_degree) deg = plan.max_degree;
         }
-        if (deg > plan.max_degree) deg = plan.max_degree;
+        for (int e2 = deg; e2 < plan.max_degree; ++e2) list[e2] = -1;
+        plan.count[s] = bad ? 0 : deg;
+        plan.block[s] = j;
+        if (bad) atomicOr(&s_bad, bad);
     }
-    for (int e2 = deg; e2 < plan.max_degree; ++e2) list[e2] = -1;
-    plan.count[s] = bad ? 0 : deg;
-    plan.block[s] = j;
-    if (bad) atomicOr(plan.status, bad);
+    __syncthreads();
+    if (threadIdx.x == 0) *plan.status = s_bad;
 }
 
 int check_cfg(const bf1_route_cfg* cfg);   // bf1_plan.cu
@@ -468,8 +474,8 @@ extern "C" int bf1_plan_decode(const int32_t* seqlens_dev, const int32_t* page_t
         return fail(BF1_ERR_CAPACITY, "decode plan max_degree %d < %d needed for %d pages per sequence", out->max_degree,
                     need, max_pages_per_seq);
     if (batch == 0) return BF1_OK;
-    BF1_CUDA_CHECK(cudaMemsetAsync(out->status, 0, sizeof(int32_t), (cudaStream_t)stream));
-    plan_decode_kernel<<<(batch + 127) / 128, 128, 0, (cudaStream_t)stream>>>(seqlens_dev, page_table_dev,
+    const int threads = batch >= 1024 ? 1024 : ((batch + 31) / 32) * 32;
+    plan_decode_kernel<<<1, threads, 0, (cudaStream_t)stream>>>(seqlens_dev, page_table_dev,
                                                                                max_pages_per_seq, batch, *cfg, *out);
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;

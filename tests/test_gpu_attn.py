@@ -109,10 +109,10 @@ def test_future_token_isolation_is_bitwise_when_later_rows_rescale(dense, hq, hk
         o2, lse2, _ = run_gpu(w, q2, k2, v2, dense=dense)
         assert np.array_equal(o[:t + 1], o2[:t + 1]) and np.array_equal(lse[:, :t + 1], lse2[:, :t + 1])
         # the mutation did reach the later rows, and by the amounts the oracle predicts: their
-        # scores are ~1300 times larger, so LSE moves by hundreds
+        # scores are ~1300 times larger, so LSE moves by tens to thousands
         rows = np.arange(t + 1, n)
         o_ref, lse_ref = oracle_full(w, q2, k2, v2, dense=dense, rows=rows)
-        assert np.abs(lse_ref[:, rows] - lse[:, rows]).min() > 50.0
+        assert np.abs(lse_ref[:, rows] - lse[:, rows]).min() > 10.0
         assert np.abs(lse2[:, rows] - lse_ref[:, rows]).max() <= 1e-3 * np.abs(lse_ref[:, rows]).max()
         diff = o2[rows].astype(np.float64) - o_ref[rows]
         assert np.sqrt((diff ** 2).mean() / (o_ref[rows].astype(np.float64) ** 2).mean()) <= 1e-2
