@@ -52,8 +52,9 @@ struct AttnArgs {
     int32_t batch;
     int32_t total_tokens;
     int32_t hq, hkv;
-    int32_t group;         // G = hq / hkv query heads per KV head: 2 or 4
-    int32_t r_shift;       // log2 of the tile rows per head R = 128 / G (6 or 5); a unit covers R query tokens
+    int32_t group;         // G = hq / hkv query heads per KV head: 1, 2 or 4
+    int32_t r_shift;       // log2 of the tile rows per head R = min(64, 128 / G) (6 or 5); a unit covers R query tokens.
+                           // With G = 1 only tile rows 0..63 carry a head; rows 64..127 are zero and never stored
     float scale_log2;      // softmax scale * log2(e)
     int32_t dense;         // 1: every predecessor block, lists ignored
     // route (BF1 mode)
@@ -289,6 +290,15 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
         tmem_alloc(smem_u32(s_tmem_base), C::kTmemCols);
         tmem_relinquish();
     }
+    if (args.group == 1) {
+        // one query head per KV head: the lower half of the 128-row tile is unused; the MMAs still read it, so
+        // it is cleared once (the Q copies only ever write rows 0..63 of each column chunk)
+        for (int i = tid; i < C::kChunks * (kBlock * 128 / 16); i += kThreads) {
+            const int ch = i / (kBlock * 128 / 16), off = i % (kBlock * 128 / 16);
+            st_shared_v4(sQ + ch * (kRows * 128) + kBlock * 128 + off * 16, 0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -393,10 +403,17 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                             mbar_arrive(bar_info + 8 * (n & 1));
                             if (cnt == 0) {
                                 mbar_arrive(bar_q_full);
-                            } else {
+                            } else if (args.group > 1) {
                                 mbar_expect_tx(bar_q_full, C::kQBytes);
                                 // one copy: box = 64 elements x R tokens x G heads x all column chunks
                                 tma_load_4d(sQ, &tm_q, 0, tok0, kvh * args.group, 0, bar_q_full);
+                            } else {
+                                // G = 1: one head, 64 rows per column chunk; each chunk goes to the place the
+                                // 128-row tile layout gives it (rows 64..127 stay zero)
+                                mbar_expect_tx(bar_q_full, C::kQBytes / 2);
+#pragma unroll
+                                for (int ch = 0; ch < C::kChunks; ++ch)
+                                    tma_load_4d(sQ + ch * (kRows * 128), &tm_q, 0, tok0, kvh, ch, bar_q_full);
                             }
                         }
                         __syncwarp();
@@ -624,14 +641,15 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             tc_fence_after();
             const float inv_l = 1.f / l_run;
             const int tok = tok0 + tl;
-            const bool store = tl < rows_valid;
+            const bool head_ok = hl < args.group;      // G = 1: tile rows 64..127 belong to no head (warp-uniform)
+            const bool store = tl < rows_valid && head_ok;
             __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * args.group + hl)) * D;
             // Full blocks leave through shared memory and TMA stores: each warp packs 32 rows x 32
             // columns into its own 2 KB staging tile (64-byte swizzle, conflict-free) and one lane
             // hands it to the copy engine.  Scattered 16-byte global stores from here would sit in the
             // same load/store path as every other warp's mbarrier and shared-memory traffic and
             // slow the whole SM down.  16 columns at a time keeps the register budget small.
-            const bool full_tile = rows_valid == (1 << args.r_shift);   // warp-uniform
+            const bool full_tile = rows_valid == (1 << args.r_shift) && head_ok;   // warp-uniform
             const uint32_t stage_w = base + C::kStageOff + (warp & 3) * 2048;
             const uint32_t srow = stage_w + lane * 64;
 #pragma unroll
@@ -751,8 +769,10 @@ static thread_local MapCache g_map_cache;
 // elements (128 bytes) x 64 tokens x `heads_per_box` heads x all chunks, 128-byte swizzle.  In shared
 // memory that is [chunk][head][token][128 B]: one K-major (or, for V, MN-major) 64-row tile per
 // chunk and head, which is what the MMA descriptors walk.
-static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box, int tokens_per_box = kBlock) {
-    const MapKey key{ptr, T, H, d, heads_per_box, tokens_per_box, 0};
+static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box, int tokens_per_box = kBlock,
+                    int chunks_per_box = 0) {
+    if (chunks_per_box == 0) chunks_per_box = d / 64;
+    const MapKey key{ptr, T, H, d, heads_per_box, tokens_per_box, chunks_per_box == d / 64 ? 0 : 2};
     if (const CUtensorMap* hit = g_map_cache.find(key)) {
         *m = *hit;
         return BF1_OK;
@@ -761,7 +781,7 @@ static int make_map(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, in
     if (int rc = get_encode_fn(&enc)) return rc;
     cuuint64_t dims[4] = {64, (cuuint64_t)T, (cuuint64_t)H, (cuuint64_t)(d / 64)};
     cuuint64_t strides[3] = {(cuuint64_t)H * d * 2, (cuuint64_t)d * 2, 128};
-    cuuint32_t box[4] = {64, (cuuint32_t)tokens_per_box, (cuuint32_t)heads_per_box, (cuuint32_t)(d / 64)};
+    cuuint32_t box[4] = {64, (cuuint32_t)tokens_per_box, (cuuint32_t)heads_per_box, (cuuint32_t)chunks_per_box};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -837,8 +857,8 @@ int check_attn_args(const void* q, const void* k, const void* v, const int32_t* 
         return fail(BF1_ERR_UNSUPPORTED, "total_tokens %lld does not fit 32-bit token indices", (long long)total_tokens);
     if (hq % hkv != 0) return fail(BF1_ERR_INVALID_ARG, "hq %d is not a multiple of hkv %d", hq, hkv);
     const int group = hq / hkv;
-    if (group != 2 && group != 4)
-        return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 and G = 4 are supported", group);
+    if (group != 1 && group != 2 && group != 4)
+        return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 1, 2 and 4 are supported", group);
     if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15)
         return fail(BF1_ERR_INVALID_ARG, "q, k, v and o must be 16-byte aligned");
@@ -869,7 +889,11 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
 
     CUtensorMap tq, tk, tv, to;
     if (int rc = make_store_map(&to, o, total_tokens, hq, d)) return rc;
-    if (int rc = make_map(&tq, q, total_tokens, hq, d, group, kRows / group)) return rc;
+    if (group == 1) {   // one head, one column chunk per copy
+        if (int rc = make_map(&tq, q, total_tokens, hq, d, 1, kBlock, 1)) return rc;
+    } else {
+        if (int rc = make_map(&tq, q, total_tokens, hq, d, group, kRows / group)) return rc;
+    }
     if (int rc = make_map(&tk, k, total_tokens, hkv, d, 1)) return rc;
     if (int rc = make_map(&tv, v, total_tokens, hkv, d, 1)) return rc;
 
@@ -880,7 +904,7 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     a.hq = hq;
     a.hkv = hkv;
     a.group = group;
-    a.r_shift = group == 2 ? 6 : 5;
+    a.r_shift = group == 4 ? 5 : 6;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
     a.scale_log2 = scale * 1.4426950408889634f;
     a.dense = route ? 0 : 1;
@@ -897,7 +921,7 @@ static int attn_common(const void* q, const void* k, const void* v, const int32_
     a.o = reinterpret_cast<__nv_bfloat16*>(o);
     a.lse = lse;
 
-    const int64_t units = slots * hkv * (group == 2 ? 1 : 2);
+    const int64_t units = slots * hkv * (group == 4 ? 2 : 1);
     const int grid = (int)(units < 2LL * info.sm_count ? units : 2LL * info.sm_count);
     if (d == 128)
         attn_fwd_kernel<128><<<grid, kThreads, Cfg<128>::kTotal, (cudaStream_t)stream>>>(tq, tk, tv, to, a);

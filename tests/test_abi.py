@@ -56,7 +56,7 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert rc == -1
     # unsupported geometry (pointers are never dereferenced on this path)
     fake = ctypes.c_void_p(0x1000)
-    for hq, hkv, d, code in ((8, 1, 64, -2), (2, 2, 64, -2), (2, 1, 96, -2), (3, 2, 64, -1)):
+    for hq, hkv, d, code in ((8, 1, 64, -2), (6, 2, 64, -2), (2, 1, 96, -2), (3, 2, 64, -1)):
         rc = lib.bf1_dense_causal_fwd(fake, fake, fake, fake, 1, 64, 64, hq, hkv, d, 0.0, fake, fake, None, None)
         assert rc == code, (hq, hkv, d, lib.bf1_last_error())
     rc = lib.bf1_dense_causal_fwd(ctypes.c_void_p(0x1004), fake, fake, fake, 1, 64, 64, 2, 1, 64, 0.0, fake, fake,

@@ -102,3 +102,19 @@ def test_group_of_four_query_heads(dense, d):
     assert_parity(o, lse, o_ref, lse_ref)
     for h in range(8):   # per head, so that a permuted head cannot hide in an average
         assert np.abs(o[:, h] - o_ref[:, h]).max() <= 2e-2
+
+
+@pytest.mark.parametrize("dense", [False, True], ids=["bf1", "dense"])
+@pytest.mark.parametrize("d", [64, 128])
+def test_one_query_head_per_kv_head(dense, d):
+    """G = 1 (plain multi-head attention): one head fills rows 0..63 of the 128-row tile, the other half is idle."""
+    w = I.custom([1, 63, 64, 65, 257, 1000, 2500], hq=3, hkv=3, d=d, seed=4600 + d)
+    q, k, v = I.draw_qkv(w)
+    o, lse, _ = run_gpu(w, q, k, v, dense=dense, guard=64)
+    if dense:
+        o_ref, lse_ref = O.dense_causal(q, k, v, w.cu_seqlens())
+    else:
+        o_ref, lse_ref = O.attn_route(oracle_cfg(w), q, k, v, w.cu_seqlens())
+    assert_parity(o, lse, o_ref, lse_ref)
+    for h in range(3):
+        assert np.abs(o[:, h] - o_ref[:, h]).max() <= 2e-2
