@@ -814,8 +814,8 @@ static int make_store_map(CUtensorMap* m, void* ptr, int64_t T, int H, int d) {
 }
 
 // the same map for the other translation units of the library
-int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box) {
-    return make_map(m, ptr, T, H, d, heads_per_box);
+int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box, int chunks_per_box) {
+    return make_map(m, ptr, T, H, d, heads_per_box, kBlock, chunks_per_box);
 }
 
 struct DeviceInfo {

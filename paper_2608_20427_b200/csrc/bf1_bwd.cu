@@ -1,4 +1,5 @@
-// BF1 attention backward (dQ, dK, dV) over the same route, for sm_100a, head dimension 128.
+// BF1 attention backward (dQ, dK, dV) over the same route, for sm_100a (head dimension 64 or 128,
+// 1, 2 or 4 query heads per KV head).
 //
 // The paper's correctness gates include a backward pass with finite Q, K and V gradients (Section
 // 4.2).  With P = exp(S - LSE) recomputed from the saved LSE and D_i = <dO_i, O_i>:
@@ -14,15 +15,17 @@
 //     dK^T = Q^T  dS          (128 x 64 x 128)   A = Q MN-major,  B = dS MN-major
 // dV^T / dK^T come out with the head dimension on the TMEM lanes; each thread adds its 64 values
 // into fp32 accumulation buffers with coalesced red.global.add.f32 (several query blocks read the
-// same KV block), and a second kernel rounds those buffers to bf16.  This first version is one CTA
-// per unit, single-buffered, every step in sequence: correctness and the operand layouts first.
+// same KV block), and a second kernel rounds those buffers to bf16.  One CTA per unit and pair of
+// query heads (G = 4: two CTAs per unit, whose dK / dV contributions meet in the fp32 buffers; G = 1:
+// the second head's rows are cleared and contribute nothing), single-buffered, every step in sequence.
+// With d = 64 the transposed products still run as M = 128 MMAs: tensor-memory lanes 64..127 then hold
+// nothing of value and are not read.
 #include <cuda.h>
 
 #include "bf1_common.cuh"
 
 namespace bf1 {
 
-constexpr int kBwdD = 128;
 constexpr int kBlock64 = 64;     // b: tokens per block
 constexpr int kBwdThreads = 128;
 
@@ -33,7 +36,7 @@ struct BwdArgs {
     const int32_t* kv_count;
     const int32_t* kv_idx;
     const int32_t* num_qblocks;
-    int32_t max_degree, capacity, total_tokens, hq, hkv;
+    int32_t max_degree, capacity, total_tokens, hq, hkv, group;
     int32_t* status;
     float scale, scale_log2;
     const __nv_bfloat16* o;
@@ -44,30 +47,35 @@ struct BwdArgs {
     float* dv32;
 };
 
+template <int D>
 struct BwdSmem {
-    static constexpr int kQ = 0;                     // Q tile   [2 chunks][128 rows][128 B]
-    static constexpr int kDO = kQ + 32768;           // dO tile  same layout
-    static constexpr int kK = kDO + 32768;           // K tile   [2 chunks][64 rows][128 B]
-    static constexpr int kV = kK + 16384;            // V tile
-    static constexpr int kP = kV;                    // P  [128 q rows][64 kv] bf16, 128-byte rows, swizzled: takes
-                                                     // over V's buffer once dP = dO V^T has been computed
+    static constexpr int kQBytes = 128 * D * 2;      // Q / dO tile [D / 64 chunks][128 rows][128 B]
+    static constexpr int kKVBytes = 64 * D * 2;      // K / V tile  [D / 64 chunks][64 rows][128 B]
+    static constexpr int kQ = 0;
+    static constexpr int kDO = kQ + kQBytes;
+    static constexpr int kK = kDO + kQBytes;
+    static constexpr int kV = kK + kKVBytes;
+    // P [128 q rows][64 kv] bf16, 128-byte rows, swizzled (16 KB).  At d = 128 it takes over V's buffer once
+    // dP = dO V^T has been computed; at d = 64 the V tile is only 8 KB, so P gets room of its own.
+    static constexpr int kP = D == 128 ? kV : kV + kKVBytes;
     static constexpr int kDS = kP + 16384;           // dS same layout
     static constexpr int kBar = kDS + 16384;
     static constexpr int kTotal = kBar + 64;
 };
 
+template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k,
                                                                const __grid_constant__ CUtensorMap tm_v,
                                                                const __grid_constant__ CUtensorMap tm_do,
                                                                const BwdArgs a) {
-    constexpr int D = kBwdD;
+    using L = BwdSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     // no static shared memory: it would cost a whole extra kilobyte and with it the second CTA per SM
-    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + BwdSmem::kBar + 32);
-    int& s_abort = *reinterpret_cast<int*>(smem + BwdSmem::kBar + 36);
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar + 32);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar + 36);
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int slot = blockIdx.x, kvh = blockIdx.y;
+    const int slot = blockIdx.x, kvh = blockIdx.y, pair = blockIdx.z;   // pair: which two query heads of the group
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
     if (slot >= min(*a.num_qblocks, a.capacity)) return;
     const int seq = a.qb_seq[slot], j = a.qb_block[slot];
@@ -79,9 +87,9 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
     const int tok0 = seq0 + j * kBlock64;
 
     const uint32_t base = smem_u32(smem);
-    const uint32_t sQ = base + BwdSmem::kQ, sDO = base + BwdSmem::kDO, sK = base + BwdSmem::kK, sV = base + BwdSmem::kV;
-    const uint32_t sP = base + BwdSmem::kP, sDS = base + BwdSmem::kDS;
-    const uint32_t bar_q = base + BwdSmem::kBar, bar_kv = bar_q + 8, bar_a = bar_q + 16, bar_b = bar_q + 24;
+    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV;
+    const uint32_t sP = base + L::kP, sDS = base + L::kDS;
+    const uint32_t bar_q = base + L::kBar, bar_kv = bar_q + 8, bar_a = bar_q + 16, bar_b = bar_q + 24;
     if (tid == 0) {
         s_abort = (base & 1023u) ? 1 : 0;
         if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
@@ -108,14 +116,33 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
 
     // rows of this thread: head hl, token tl of the query block
     const int hl = tid >> 6, tl = tid & 63;
-    const int h = kvh * 2 + hl;
+    const int h = kvh * a.group + pair * 2 + hl;
     const int tok = tok0 + tl;
-    const bool row_ok = tl < rows_valid;
+    const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;   // G = 1: rows 64..127 belong to no head
 
+    if (a.group == 1) {
+        // one head: rows 64..127 of every column chunk of the Q and dO tiles are never written by a copy; the
+        // MMAs still read them, so they are cleared (they then give P = 0 and dS = 0 like rows past a sequence)
+        for (int i = tid; i < 2 * (D / 64) * 512; i += kBwdThreads) {
+            const int which = i / ((D / 64) * 512), ch = (i / 512) % (D / 64), off = i % 512;
+            st_shared_v4((which ? sDO : sQ) + ch * 16384 + 8192 + off * 16, 0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async();
+        __syncthreads();
+    }
     if (tid == 0 && !s_abort) {
-        mbar_expect_tx(bar_q, 65536);
-        tma_load_4d(sQ, &tm_q, 0, tok0, kvh * 2, 0, bar_q);
-        tma_load_4d(sDO, &tm_do, 0, tok0, kvh * 2, 0, bar_q);
+        if (a.group > 1) {
+            mbar_expect_tx(bar_q, 2 * L::kQBytes);
+            tma_load_4d(sQ, &tm_q, 0, tok0, h, 0, bar_q);      // h: the pair's first head (hl = 0 here)
+            tma_load_4d(sDO, &tm_do, 0, tok0, h, 0, bar_q);
+        } else {
+            mbar_expect_tx(bar_q, L::kQBytes);                 // 64 rows of each
+#pragma unroll
+            for (int ch = 0; ch < D / 64; ++ch) {
+                tma_load_4d(sQ + ch * 16384, &tm_q, 0, tok0, h, ch, bar_q);
+                tma_load_4d(sDO + ch * 16384, &tm_do, 0, tok0, h, ch, bar_q);
+            }
+        }
     }
     // D_i = <dO_i, O_i> and the row's LSE in the log2 domain
     float Drow = 0.f, lse2 = 0.f;
@@ -151,7 +178,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
         return p;
     };
     auto load_kv = [&](int p) {   // thread 0 only
-        mbar_expect_tx(bar_kv, 32768);
+        mbar_expect_tx(bar_kv, 2 * L::kKVBytes);
         tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
         tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
     };
@@ -230,7 +257,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
             // dQ += dS K: A = dS [128 q][64 kv] K-major (4 k-steps of 16 kv = 32 bytes), B = K tile MN-major
             // (16 kv rows = 2048 bytes per step, next 64 d columns 8 KB away)
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
+            for (int kk = 0; kk < 4; ++kk) {   // 64 kv rows in steps of 16
                 const uint32_t alo = desc_lo_sw128(sDS, 16) + ((kk * 32) >> 4);
                 const uint32_t blo = desc_lo_sw128(sK, 8192) + ((kk * 2048) >> 4);
                 if (it == 0 && kk == 0) mma_ss_lohi<false>(tmem + kColDQ, alo, blo, kHi, kIdQ);
@@ -261,6 +288,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
         float* dvp = a.dv32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
         float* dkp = a.dk32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
         const size_t rstride = (size_t)a.hkv * D;
+        const bool lane_ok = tid < D;   // d = 64: lanes 64..127 of the transposed products hold nothing (warp-uniform)
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             uint32_t vr[32], kr[32];
@@ -270,7 +298,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
                 const int kvr = half * 32 + c;
-                if (kvr < kv_valid) {
+                if (kvr < kv_valid && lane_ok) {
                     atomicAdd(dvp + kvr * rstride, __uint_as_float(vr[c]));
                     atomicAdd(dkp + kvr * rstride, __uint_as_float(kr[c]));
                 }
@@ -315,7 +343,7 @@ __global__ void bwd_round_kernel(const float* __restrict__ src_k, const float* _
     }
 }
 
-int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box);   // bf1_attn.cu
+int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box, int chunks_per_box);   // bf1_attn.cu
 
 }  // namespace bf1
 
@@ -336,8 +364,10 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
         return fail(BF1_ERR_INVALID_ARG, "negative or zero size argument");
     if (total_tokens > 0x7fffffffLL - 64) return fail(BF1_ERR_UNSUPPORTED, "total_tokens does not fit 32-bit token indices");
     if (hq % hkv != 0) return fail(BF1_ERR_INVALID_ARG, "hq %d is not a multiple of hkv %d", hq, hkv);
-    if (hq / hkv != 2) return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 is supported", hq / hkv);
-    if (d != 128) return fail(BF1_ERR_UNSUPPORTED, "backward: head dimension %d: only 128 is supported", d);
+    const int group = hq / hkv;
+    if (group != 1 && group != 2 && group != 4)
+        return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 1, 2 and 4 are supported", group);
+    if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o | (uintptr_t)d_o | (uintptr_t)dq | (uintptr_t)dk |
          (uintptr_t)dv | (uintptr_t)workspace) & 15)
         return fail(BF1_ERR_INVALID_ARG, "tensors and workspace must be 16-byte aligned");
@@ -350,15 +380,20 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     BF1_CUDA_CHECK(cudaGetDevice(&dev));
     BF1_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
     if (major != 10) return fail(BF1_ERR_NO_DEVICE, "device compute capability %d.x is not sm_100", major);
-    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem::kTotal));
+    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal));
+    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal));
     // two CTAs per SM need the whole shared-memory carve-out
-    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared));
+    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                         cudaSharedmemCarveoutMaxShared));
     CUtensorMap tq, tk, tv, tg;
-    if (int rc = make_map_4d(&tq, q, total_tokens, hq, d, 2)) return rc;
-    if (int rc = make_map_4d(&tg, d_o, total_tokens, hq, d, 2)) return rc;
-    if (int rc = make_map_4d(&tk, k, total_tokens, hkv, d, 1)) return rc;
-    if (int rc = make_map_4d(&tv, v, total_tokens, hkv, d, 1)) return rc;
+    // Q and dO: two heads and all column chunks per copy; with one head per KV head, one head and one chunk
+    const int q_heads = group == 1 ? 1 : 2, q_chunks = group == 1 ? 1 : d / 64;
+    if (int rc = make_map_4d(&tq, q, total_tokens, hq, d, q_heads, q_chunks)) return rc;
+    if (int rc = make_map_4d(&tg, d_o, total_tokens, hq, d, q_heads, q_chunks)) return rc;
+    if (int rc = make_map_4d(&tk, k, total_tokens, hkv, d, 1, d / 64)) return rc;
+    if (int rc = make_map_4d(&tv, v, total_tokens, hkv, d, 1, d / 64)) return rc;
     const size_t n_kv = (size_t)total_tokens * hkv * d;
     BwdArgs a;
     a.cu_seqlens = cu_seqlens_dev;
@@ -372,6 +407,7 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.total_tokens = (int32_t)total_tokens;
     a.hq = hq;
     a.hkv = hkv;
+    a.group = group;
     a.status = route->status;
     a.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
     a.scale_log2 = a.scale * 1.4426950408889634f;
@@ -383,8 +419,9 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.dv32 = a.dk32 + n_kv;
     cudaStream_t st = (cudaStream_t)stream;
     BF1_CUDA_CHECK(cudaMemsetAsync(workspace, 0, 2 * n_kv * sizeof(float), st));
-    dim3 grid(route->capacity_qblocks, hkv);
-    attn_bwd_kernel<<<grid, kBwdThreads, BwdSmem::kTotal, st>>>(tq, tk, tv, tg, a);
+    dim3 grid(route->capacity_qblocks, hkv, group == 4 ? 2 : 1);   // z: pairs of query heads
+    if (d == 128) attn_bwd_kernel<128><<<grid, kBwdThreads, BwdSmem<128>::kTotal, st>>>(tq, tk, tv, tg, a);
+    else attn_bwd_kernel<64><<<grid, kBwdThreads, BwdSmem<64>::kTotal, st>>>(tq, tk, tv, tg, a);
     BF1_CUDA_CHECK(cudaGetLastError());
     bwd_round_kernel<<<296, 512, 0, st>>>(a.dk32, a.dv32, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_kv);
     BF1_CUDA_CHECK(cudaGetLastError());

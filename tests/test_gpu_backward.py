@@ -78,13 +78,32 @@ def test_gradients_at_the_benchmarked_lengths(n):
         assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
 
 
-def test_backward_rejects_head_dim_64():
+@pytest.mark.parametrize("hq,hkv,d", [(4, 2, 64), (8, 2, 128), (8, 2, 64), (3, 3, 128), (2, 2, 64)],
+                         ids=["G2-d64", "G4-d128", "G4-d64", "G1-d128", "G1-d64"])
+def test_gradients_in_every_geometry_the_forward_takes(hq, hkv, d):
+    """Section 4.2's gradient gate per geometry: head dimension 64, four query heads per KV head (two CTAs per unit
+    whose dK / dV contributions add up), one query head per KV head (half of the tile idle)."""
+    for lens in ([1, 65, 257, 1000], [2500]):
+        w = I.custom(lens, hq=hq, hkv=hkv, d=d, seed=6300 + hq + d + len(lens))
+        res = run_case(w, seed=4)
+        print(hq, hkv, d, lens, res)
+        for name, (rms, mx) in res.items():
+            assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
+
+
+def test_backward_rejects_what_it_does_not_support():
     dev = torch.device("cuda:0")
     w = I.custom([128], hq=2, hkv=1, d=64, seed=1)
     q, k, v = (t.to(dev) for t in I.draw_qkv(w))
     cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
     route = bf1.plan_route(cu, 128)
     o, lse = bf1.attn_fwd(q, k, v, cu, 128, route)
-    with pytest.raises(bf1.Bf1Error) as e:
-        bf1.attn_bwd(q, k, v, o, lse, torch.zeros_like(q), cu, 128, route)
-    assert e.value.code == -2
+    lib = bf1.load()
+    rc = lib.bf1_attn_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), q.data_ptr(),
+                          cu.data_ptr(), 1, 128, 128, 6, 1, 64, 0.0, route.c, q.data_ptr(), q.data_ptr(), q.data_ptr(),
+                          q.data_ptr(), None)
+    assert rc == -2 and b"group" in lib.bf1_last_error()      # G = 6
+    rc = lib.bf1_attn_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), q.data_ptr(),
+                          cu.data_ptr(), 1, 128, 128, 2, 1, 96, 0.0, route.c, q.data_ptr(), q.data_ptr(), q.data_ptr(),
+                          q.data_ptr(), None)
+    assert rc == -2 and b"dimension" in lib.bf1_last_error()  # d = 96
