@@ -421,7 +421,7 @@ def decode_sweep(bf1, dev):
             sl = torch.full((batch,), n, dtype=torch.int32, device=dev)
             tables = [torch.randint(0, pool, (batch, nb), generator=g, device=dev, dtype=torch.int32) for _ in range(reps)]
             plans = [bf1.plan_decode(sl, t) for t in tables]
-            ws = bf1.decode_workspace(batch, hkv, plans[0].max_degree, d, dev)
+            ws = bf1.decode_workspace(batch, hq, hkv, plans[0].max_degree, d, dev)
             o = torch.empty_like(q)
             lse = torch.empty((hq, batch), dtype=torch.float32, device=dev)
             torch.cuda.synchronize()
@@ -469,7 +469,7 @@ def run_single_decode(args, bf1, dev):
     total = args.warmup + args.steps
     tables = [torch.randint(0, pool, (batch, n // 64), generator=g, device=dev, dtype=torch.int32) for _ in range(total)]
     plans = [bf1.plan_decode(sl, t) for t in tables]
-    ws = bf1.decode_workspace(batch, hkv, plans[0].max_degree, d, dev)
+    ws = bf1.decode_workspace(batch, hq, hkv, plans[0].max_degree, d, dev)
     o = torch.empty_like(q)
     lse = torch.empty((hq, batch), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()

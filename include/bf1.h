@@ -198,8 +198,9 @@ int bf1_plan_decode(const int32_t *seqlens_dev, const int32_t *page_table_dev,
                     const bf1_decode_plan *out /* host struct, device arrays */, void *stream);
 
 /* Bytes of device scratch bf1_decode_fwd needs (partial results of the split over pages and one
- * ticket word per sequence and KV head).  Host only; -1 on bad arguments. */
-int64_t bf1_decode_workspace_bytes(int32_t batch, int32_t hkv, int32_t max_degree, int32_t d);
+ * ticket word per sequence, KV head and pair of query heads).  Host only; -1 on bad arguments. */
+int64_t bf1_decode_workspace_bytes(int32_t batch, int32_t hq, int32_t hkv, int32_t max_degree,
+                                   int32_t d);
 
 /* One decode step for every sequence of the batch.
  *   q            device bf16 [batch, hq, d]: the newest token's queries

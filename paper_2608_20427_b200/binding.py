@@ -79,7 +79,7 @@ def load():
     L.bf1_plan_decode.restype = ctypes.c_int
     L.bf1_plan_decode.argtypes = [vp, vp, i32, i32, ctypes.POINTER(RouteCfg), ctypes.POINTER(_DecodePlanC), vp]
     L.bf1_decode_workspace_bytes.restype = i64
-    L.bf1_decode_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.bf1_decode_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     L.bf1_decode_fwd.restype = ctypes.c_int
     L.bf1_decode_fwd.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, f32, ctypes.POINTER(_DecodePlanC), vp, vp,
                                  vp, vp]
@@ -281,9 +281,9 @@ def plan_decode(seqlens: torch.Tensor, page_table: torch.Tensor, cfg: Optional[R
     return plan
 
 
-def decode_workspace(batch: int, hkv: int, max_degree: int, d: int, device) -> torch.Tensor:
+def decode_workspace(batch: int, hq: int, hkv: int, max_degree: int, d: int, device) -> torch.Tensor:
     """Zero-initialised scratch for decode_fwd (reusable across calls that do not overlap)."""
-    nbytes = int(load().bf1_decode_workspace_bytes(batch, hkv, max_degree, d))
+    nbytes = int(load().bf1_decode_workspace_bytes(batch, hq, hkv, max_degree, d))
     return torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
 
 

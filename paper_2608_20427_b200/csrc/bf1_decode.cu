@@ -33,9 +33,10 @@ struct DecodeArgs {
     const int32_t* block;             // plan: [batch] block index the plan was made for
     int32_t* status;
     int32_t max_degree, hq, hkv, num_pages;
+    int32_t group, pairs;             // G = hq / hkv (1, 2 or 4) and ceil(G / 2): a CTA serves one pair of query heads
     float scale_log2;
-    float* part;                      // [batch, hkv, max_degree, 2, d + 2] partial (o[d], m, l)
-    int32_t* ticket;                  // [batch, hkv], zero before and after every call
+    float* part;                      // [batch, hkv * pairs, max_degree, 2, d + 2] partial (o[d], m, l)
+    int32_t* ticket;                  // [batch, hkv * pairs], zero before and after every call
     __nv_bfloat16* o;                 // [batch, hq, d]
     float* lse;                       // [hq, batch]
     int32_t batch;
@@ -56,7 +57,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
     __shared__ float sW[2][64];                         // combine: weight of every partial
     __shared__ int sLast;
 
-    const int e = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
+    const int e = blockIdx.x, kvp = blockIdx.y, s = blockIdx.z;
+    const int kvh = kvp / a.pairs, hbase = kvh * a.group + (kvp % a.pairs) * 2;   // first query head of this CTA's pair
+    const int nheads = min(2, a.group - (kvp % a.pairs) * 2);                      // 1 when G = 1
     const int tid = threadIdx.x;
     // the four scalars this CTA needs are independent loads: issue them together
     const int cnt = a.count[s];
@@ -66,7 +69,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
     if (e >= cnt) return;
     const int j = (n - 1) / kPage;
     if (j != planned) {               // the plan belongs to another route epoch
-        if (tid == 0 && e == 0 && kvh == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+        if (tid == 0 && e == 0 && kvp == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
         return;
     }
     if (pg < 0 || pg >= a.num_pages) {
@@ -89,7 +92,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
             vreg[it] = *reinterpret_cast<const uint4*>(vp + r * row_stride + c * 8);
         }
         for (int i = tid; i < 2 * D; i += kDecThreads)
-            sQ[i / D][i % D] = __bfloat162float(a.q[((size_t)s * a.hq + kvh * 2 + i / D) * D + i % D]);
+            sQ[i / D][i % D] = i / D < nheads ? __bfloat162float(a.q[((size_t)s * a.hq + hbase + i / D) * D + i % D]) : 0.f;
 #pragma unroll
         for (int it = 0; it < kVecPerThread; ++it) {
             const int i = tid + it * kDecThreads, r = i / kVecPerRow, c = i % kVecPerRow;
@@ -155,7 +158,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
 #pragma unroll 8
         for (int k = 0; k < valid; ++k) acc[0] = fmaf(sP[h][k], __bfloat162float(sVh[k * D + c0]), acc[0]);
     }
-    float* my = a.part + ((((size_t)s * a.hkv + kvh) * a.max_degree + e) * 2 + h) * (D + 2);
+    float* my = a.part + ((((size_t)s * a.hkv * a.pairs + kvp) * a.max_degree + e) * 2 + h) * (D + 2);
 #pragma unroll
     for (int c = 0; c < kColsPerThread; ++c) my[c0 + c] = acc[c];
     if (r == 0) { my[D] = mx; my[D + 1] = sum; }
@@ -164,14 +167,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const int t = atomicAdd(a.ticket + s * a.hkv + kvh, 1);
+        const int t = atomicAdd(a.ticket + s * a.hkv * a.pairs + kvp, 1);
         sLast = (t == cnt - 1);
-        if (sLast) a.ticket[s * a.hkv + kvh] = 0;        // ready for the next call
+        if (sLast) a.ticket[s * a.hkv * a.pairs + kvp] = 0;   // ready for the next call
     }
     __syncthreads();
     if (!sLast) return;
     __threadfence();
-    const float* base = a.part + (((size_t)s * a.hkv + kvh) * a.max_degree * 2 + h) * (D + 2);
+    const float* base = a.part + (((size_t)s * a.hkv * a.pairs + kvp) * a.max_degree * 2 + h) * (D + 2);
     const size_t estride = 2 * (D + 2);
     // every partial's (max, sum) is fetched by its own thread, so the loads overlap
     if (r < cnt) sW[h][r] = base[r * estride + D];
@@ -198,11 +201,12 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a)
 #pragma unroll
         for (int c = 0; c < kColsPerThread; ++c) out[c] = fmaf(w, base[i * estride + c0 + c], out[c]);
     }
+    if (h >= nheads) return;                             // G = 1: the second head of the pair does not exist
     const float inv = 1.f / l_all;
-    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + kvh * 2 + h) * D;
+    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + hbase + h) * D;
 #pragma unroll
     for (int c = 0; c < kColsPerThread; ++c) orow[c0 + c] = __float2bfloat16_rn(out[c] * inv);
-    if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+    if (r == 0) a.lse[(size_t)(hbase + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -251,14 +255,16 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
     __shared__ float sM[4][2], sL[4][2];
     __shared__ float sO[4][2][D];
 
-    const int kvh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
+    const int kvp = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
+    const int kvh = kvp / a.pairs, hbase = kvh * a.group + (kvp % a.pairs) * 2;   // first query head of this CTA's pair
+    const int nheads = min(2, a.group - (kvp % a.pairs) * 2);                      // 1 when G = 1
     const int warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
     const int cnt = a.count[s];
     const int n = a.seqlens[s];
     if (cnt <= 0) return;
     const int j = (n - 1) / kPage;
     if (j != a.block[s]) {            // the plan belongs to another route epoch
-        if (tid == 0 && kvh == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
+        if (tid == 0 && kvp == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
         return;
     }
     const int tail = n - j * kPage;   // valid tokens of the self page (the last list entry)
@@ -291,11 +297,11 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
     // A fragments of Q: rows 0 and 1 of the 16-row operand are the two grouped heads, the rest zero
     uint32_t qa[D / 16][2];
     {
-        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + ((size_t)s * a.hq + kvh * 2 + (gid & 1)) * D);
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + ((size_t)s * a.hq + hbase + (gid < nheads ? gid : 0)) * D);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-            qa[kk][0] = gid < 2 ? qrow[kk * 8 + tig] : 0u;          // columns kk*16 + 2*tig, +1
-            qa[kk][1] = gid < 2 ? qrow[kk * 8 + tig + 4] : 0u;      // columns kk*16 + 8 + 2*tig, +1
+            qa[kk][0] = gid < nheads ? qrow[kk * 8 + tig] : 0u;          // columns kk*16 + 2*tig, +1
+            qa[kk][1] = gid < nheads ? qrow[kk * 8 + tig + 4] : 0u;      // columns kk*16 + 8 + 2*tig, +1
         }
     }
     float m_run = -INFINITY, l_run = 0.f;                // per lane: head gid (lanes with gid >= 2 carry dummies)
@@ -386,9 +392,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         wgt[w] = exp2f(sM[w][h] - m_all);                // 0 for a warp that never saw a valid key
         l_all = fmaf(wgt[w], sL[w][h], l_all);
     }
+    if (h >= nheads) return;                             // G = 1: the second head of the pair does not exist
     const float inv = 1.f / l_all;
     constexpr int kColsPerThread = D / 64;
-    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + kvh * 2 + h) * D;
+    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + hbase + h) * D;
 #pragma unroll
     for (int c = 0; c < kColsPerThread; ++c) {
         const int col = r * kColsPerThread + c;
@@ -397,7 +404,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         for (int w = 0; w < 4; ++w) o = fmaf(wgt[w], sO[w][h][col], o);
         orow[col] = __float2bfloat16_rn(o * inv);
     }
-    if (r == 0) a.lse[(size_t)(kvh * 2 + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+    if (r == 0) a.lse[(size_t)(hbase + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
 // One thread per sequence: Eq. 1 for the block of the newest token, mapped through the page table.
@@ -453,10 +460,11 @@ int check_cfg(const bf1_route_cfg* cfg);   // bf1_plan.cu
 
 using namespace bf1;
 
-extern "C" int64_t bf1_decode_workspace_bytes(int32_t batch, int32_t hkv, int32_t max_degree, int32_t d) {
-    if (batch < 0 || hkv <= 0 || max_degree <= 0 || d <= 0) return -1;
-    const int64_t part = (int64_t)batch * hkv * max_degree * 2 * (d + 2) * (int64_t)sizeof(float);
-    const int64_t tick = (int64_t)batch * hkv * (int64_t)sizeof(int32_t);
+extern "C" int64_t bf1_decode_workspace_bytes(int32_t batch, int32_t hq, int32_t hkv, int32_t max_degree, int32_t d) {
+    if (batch < 0 || hq <= 0 || hkv <= 0 || hq % hkv != 0 || max_degree <= 0 || d <= 0) return -1;
+    const int64_t pairs = (hq / hkv + 1) / 2;   // CTAs (and partial-result slots) per KV head
+    const int64_t part = (int64_t)batch * hkv * pairs * max_degree * 2 * (d + 2) * (int64_t)sizeof(float);
+    const int64_t tick = (int64_t)batch * hkv * pairs * (int64_t)sizeof(int32_t);
     return ((part + 255) / 256) * 256 + tick;
 }
 
@@ -491,11 +499,13 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
         return fail(BF1_ERR_INVALID_ARG, "a decode-plan pointer is null");
     if (batch < 0 || num_pages < 0 || hq <= 0 || hkv <= 0) return fail(BF1_ERR_INVALID_ARG, "negative or zero size argument");
     if (hq % hkv != 0) return fail(BF1_ERR_INVALID_ARG, "hq %d is not a multiple of hkv %d", hq, hkv);
-    if (hq / hkv != 2) return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 2 is supported", hq / hkv);
+    const int group = hq / hkv, pairs = (group + 1) / 2;
+    if (group != 1 && group != 2 && group != 4)
+        return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 1, 2 and 4 are supported", group);
     if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)o | (uintptr_t)workspace) & 15)
         return fail(BF1_ERR_INVALID_ARG, "q, k_pages, v_pages, o and workspace must be 16-byte aligned");
-    if (plan->max_degree < 1 || plan->max_degree > 64 || hkv > 65535 || batch > 65535)
+    if (plan->max_degree < 1 || plan->max_degree > 64 || hkv * pairs > 65535 || batch > 65535)
         return fail(BF1_ERR_UNSUPPORTED, "max_degree must be <= 64; hkv and batch must fit the grid (<= 65535)");
     if (batch == 0) return BF1_OK;
     DecodeArgs a;
@@ -511,10 +521,12 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
     a.hq = hq;
     a.hkv = hkv;
     a.num_pages = num_pages;
+    a.group = group;
+    a.pairs = pairs;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
     a.scale_log2 = scale * 1.4426950408889634f;
     a.part = (float*)workspace;
-    const int64_t part = (int64_t)batch * hkv * plan->max_degree * 2 * (d + 2) * (int64_t)sizeof(float);
+    const int64_t part = (int64_t)batch * hkv * pairs * plan->max_degree * 2 * (d + 2) * (int64_t)sizeof(float);
     a.ticket = (int32_t*)((char*)workspace + ((part + 255) / 256) * 256);
     a.o = (__nv_bfloat16*)o;
     a.lse = lse;
@@ -528,14 +540,14 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
         BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 64 * 2));
         BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     }
-    if ((int64_t)batch * hkv >= sm_count[dev]) {
+    if ((int64_t)batch * hkv * pairs >= sm_count[dev]) {
         // enough (sequence, KV head) pairs to fill the GPU: one CTA walks a whole list
-        dim3 grid(hkv, batch);
+        dim3 grid(hkv * pairs, batch);
         if (d == 128) decode_fused_kernel<128><<<grid, kDecThreads, kDecStages * 2 * 64 * 128 * 2, (cudaStream_t)stream>>>(a);
         else decode_fused_kernel<64><<<grid, kDecThreads, kDecStages * 2 * 64 * 64 * 2, (cudaStream_t)stream>>>(a);
     } else {
         // few pairs: split every list over CTAs (one page each) and combine
-        dim3 grid(plan->max_degree, hkv, batch);
+        dim3 grid(plan->max_degree, hkv * pairs, batch);
         if (d == 128) decode_kernel<128><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
         else decode_kernel<64><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
     }

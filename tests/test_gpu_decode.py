@@ -49,13 +49,14 @@ def run_decode(w, q, k_pages, v_pages, table, seqlens=None, plan=None):
     tb = table.to(dev)
     if plan is None:
         plan = bf1.plan_decode(sl, tb)
-    ws = bf1.decode_workspace(len(w.seqlens), w.hkv, plan.max_degree, w.d, dev)
+    ws = bf1.decode_workspace(len(w.seqlens), w.hq, w.hkv, plan.max_degree, w.d, dev)
     out = torch.full((len(w.seqlens), w.hq, w.d), float("nan"), dtype=torch.bfloat16, device=dev)
     lse = torch.full((w.hq, len(w.seqlens)), float("nan"), dtype=torch.float32, device=dev)
     for _ in range(2):   # twice: the second call finds the ticket words the first one left
         bf1.decode_fwd(qd, k_pages.to(dev), v_pages.to(dev), sl, plan, ws, out=out, lse=lse)
     torch.cuda.synchronize()
-    assert int(ws.view(torch.int32)[-len(w.seqlens) * w.hkv:].abs().sum().item()) == 0
+    pairs = (w.hq // w.hkv + 1) // 2
+    assert int(ws.view(torch.int32)[-len(w.seqlens) * w.hkv * pairs:].abs().sum().item()) == 0
     return out.float().cpu().numpy(), lse.cpu().numpy(), plan, last
 
 
@@ -175,7 +176,7 @@ def test_one_plan_serves_a_route_epoch_and_refuses_the_next():
         check(wn, q[:n], k[:n], v[:n], out, lse, last)
     # one token further the newest token lives in block 10: the stale plan is flagged, nothing is read
     dev_sl = torch.tensor([n0 + 64], dtype=torch.int32, device=dev)
-    ws = bf1.decode_workspace(1, 2, plan.max_degree, 128, dev)
+    ws = bf1.decode_workspace(1, 4, 2, plan.max_degree, 128, dev)
     bf1.decode_fwd(q[:1].to(dev), k_pages.to(dev), v_pages.to(dev), dev_sl, plan, ws)
     torch.cuda.synchronize()
     assert int(plan.status.item()) & 8
@@ -187,3 +188,17 @@ def test_decode_plan_flags_a_sequence_longer_than_its_page_table():
     plan = bf1.plan_decode(torch.tensor([4 * 64 + 1], dtype=torch.int32, device=dev), table)
     torch.cuda.synchronize()
     assert int(plan.status.item()) & 1 and int(plan.count.item()) == 0
+
+
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (3, 3)], ids=["G4", "G1"])
+@pytest.mark.parametrize("batch_kind", ["few", "many"])
+def test_decode_with_four_and_with_one_query_head_per_kv_head(hq, hkv, batch_kind):
+    """G = 4 runs two CTAs (pairs of query heads) per KV head, G = 1 half a pair; both the split kernel
+    (few sequences) and the one-CTA-per-list kernel (many) are exercised."""
+    lens = [1, 64, 65, 257, 1000, 0, 4097] if batch_kind == "few" else [1 + (37 * i) % 700 for i in range(90)]
+    w = I.custom(lens, hq=hq, hkv=hkv, d=128, seed=7100 + hq + len(lens))
+    q, k, v = I.draw_qkv(w)
+    k_pages, v_pages, table = paged_cache(w, k, v, seed=7200 + hq)
+    out, lse, plan, last = run_decode(w, q, k_pages, v_pages, table)
+    assert int(plan.status.item()) == 0
+    check(w, q, k, v, out, lse, last)
