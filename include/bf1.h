@@ -231,6 +231,35 @@ int bf1_attn_bwd(const void *q, const void *k, const void *v, const void *o, con
                  const bf1_route *route /* host */, void *workspace, void *dq, void *dk, void *dv,
                  void *stream);
 
+/* ---- sequence-sharded prefill ----------------------------------------------------------------------
+ * One long sequence cut into contiguous shards of whole blocks, one shard per GPU.  The route is
+ * "block aligned and data independent" (Section 3.1), so the KV blocks a shard reads from earlier shards
+ * -- block 0, the two blocks in front of it, and the dyadic predecessors j - 2^k of its query blocks
+ * that fall in front of it: O(shard blocks x log B) blocks, Proposition 1 -- are known at plan time,
+ * before any tensor exists.  The exchange itself is left to the caller's communication library (plain
+ * point-to-point copies into a landing buffer in the receiver's own memory); the library provides the
+ * two plans:
+ *
+ * bf1_shard_needed_blocks (host only): the ascending global indices of the KV blocks that the shard
+ * of query blocks [lo_block, hi_block) reads but does not own (all are < lo_block).  Returns
+ * BF1_ERR_CAPACITY when `capacity` entries are not enough (count_out still receives the number).
+ *
+ * bf1_plan_route_shard (device): the shard's route over its LOCAL key/value tensor, which the caller
+ * lays out as [the needed blocks in ascending global order | the shard's own blocks], 64 token rows
+ * per block ("virtual sequence").  Query, output and LSE tensors use the same row numbering (their
+ * first num_needed * 64 rows are never touched).  Lists are re-indexed into that layout: entries stay
+ * ascending and end in the query block itself, so bf1_attn_fwd runs the shard unchanged, with
+ * cu_seqlens_out_dev = {0, num_needed * 64 + the shard's tokens} written by this call.  Counts and
+ * totals are the shard's share of the sequence's selected pairs.  A block of some list that is
+ * neither owned nor in `needed_blocks_dev` sets BF1_DEV_BAD_ROUTE in *out->status. */
+int bf1_shard_needed_blocks(int64_t n_tokens, const bf1_route_cfg *cfg /* host */, int32_t lo_block,
+                            int32_t hi_block, int32_t *blocks_out /* host */, int32_t capacity,
+                            int32_t *count_out /* host */);
+int bf1_plan_route_shard(int64_t n_tokens, int32_t lo_block, int32_t hi_block,
+                         const bf1_route_cfg *cfg /* host */, const int32_t *needed_blocks_dev,
+                         int32_t num_needed, const bf1_route *out /* host struct, device arrays */,
+                         int32_t *cu_seqlens_out_dev /* [2] */, void *stream);
+
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char *bf1_last_error(void);
 

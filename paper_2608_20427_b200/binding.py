@@ -20,7 +20,8 @@ DEV_BAD_SEQLENS, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_ROUTE = 1, 2, 4, 8
 
 EXPORTS = ("bf1_route_capacity", "bf1_plan_route", "bf1_attn_fwd", "bf1_dense_causal_fwd",
            "bf1_attn_fwd_noalloc", "bf1_plan_decode", "bf1_decode_workspace_bytes", "bf1_decode_fwd",
-           "bf1_attn_bwd", "bf1_attn_bwd_workspace_bytes", "bf1_last_error", "bf1_version")
+           "bf1_attn_bwd", "bf1_attn_bwd_workspace_bytes", "bf1_shard_needed_blocks", "bf1_plan_route_shard",
+           "bf1_last_error", "bf1_version")
 
 
 class RouteCfg(ctypes.Structure):
@@ -88,6 +89,10 @@ def load():
     L.bf1_attn_bwd.restype = ctypes.c_int
     L.bf1_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(_RouteC),
                                vp, vp, vp, vp, vp]
+    L.bf1_shard_needed_blocks.restype = ctypes.c_int
+    L.bf1_shard_needed_blocks.argtypes = [i64, ctypes.POINTER(RouteCfg), i32, i32, ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
+    L.bf1_plan_route_shard.restype = ctypes.c_int
+    L.bf1_plan_route_shard.argtypes = [i64, i32, i32, ctypes.POINTER(RouteCfg), vp, i32, ctypes.POINTER(_RouteC), vp, vp]
     L.bf1_last_error.restype = ctypes.c_char_p
     L.bf1_last_error.argtypes = []
     L.bf1_version.restype = ctypes.c_int
@@ -317,6 +322,35 @@ def attn_bwd(q, k, v, o, lse, d_o, cu_seqlens, max_seqlen: int, route: Route, sc
                                float(scale) if scale else 0.0, ctypes.byref(route.c), workspace.data_ptr(),
                                dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), _stream_ptr(stream)))
     return dq, dk, dv
+
+
+def shard_needed_blocks(n_tokens: int, lo_block: int, hi_block: int, cfg: Optional[RouteCfg] = None):
+    """bf1_shard_needed_blocks: ascending global KV blocks the shard [lo_block, hi_block) reads but does not own (host only)."""
+    cfg = cfg or RouteCfg()
+    cap = max(lo_block, 1)
+    buf = (ctypes.c_int32 * cap)()
+    count = ctypes.c_int32(0)
+    _check(load().bf1_shard_needed_blocks(n_tokens, ctypes.byref(cfg), lo_block, hi_block, buf, cap, ctypes.byref(count)))
+    return list(buf[:count.value])
+
+
+def plan_route_shard(n_tokens: int, lo_block: int, hi_block: int, needed_blocks: torch.Tensor,
+                     cfg: Optional[RouteCfg] = None, route: Optional[Route] = None, stream=None):
+    """bf1_plan_route_shard: the shard's route over its local [needed | own] key/value tensor.
+    Returns (route, cu_seqlens [2] int32 device tensor of the shard's virtual sequence)."""
+    cfg = cfg or RouteCfg()
+    assert needed_blocks.dtype == torch.int32 and needed_blocks.is_cuda
+    if route is None:
+        _, deg = route_capacity(1, n_tokens, n_tokens, cfg)
+        route = Route.empty(hi_block - lo_block, deg, needed_blocks.device, cfg)
+    cu = torch.zeros(2, dtype=torch.int32, device=needed_blocks.device)
+    _check(load().bf1_plan_route_shard(n_tokens, lo_block, hi_block, ctypes.byref(cfg),
+                                       needed_blocks.data_ptr() if needed_blocks.numel() else None, needed_blocks.numel(),
+                                       ctypes.byref(route.c), cu.data_ptr(), _stream_ptr(stream)))
+    own_tokens = min(n_tokens, hi_block * 64) - lo_block * 64
+    cu._bf1_total = needed_blocks.numel() * 64 + own_tokens
+    route.cfg = cfg
+    return route, cu
 
 
 def cu_seqlens_tensor(seqlens: Sequence[int], device) -> torch.Tensor:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbf1.so")
-SOURCES = ["bf1_plan.cu", "bf1_attn.cu", "bf1_noalloc.cu", "bf1_decode.cu", "bf1_bwd.cu"]
+SOURCES = ["bf1_plan.cu", "bf1_attn.cu", "bf1_noalloc.cu", "bf1_decode.cu", "bf1_bwd.cu", "bf1_shard.cu"]
 HEADERS = ["bf1_common.cuh", os.path.join("..", "..", "include", "bf1.h")]
 
 
