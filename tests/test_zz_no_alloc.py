@@ -39,7 +39,7 @@ def test_requests_beyond_the_built_in_scratch_are_refused_on_the_host():
                                   fake, fake, None, None)
     assert rc == -3 and b"32" in lib.bf1_last_error()
     # geometry and pointer errors come before the capacity check and before anything is launched
-    rc = lib.bf1_attn_fwd_noalloc(fake, fake, fake, fake, 1, n, n, 16, 16, 128, 0.0, ctypes.byref(cfg), fake, fake,
+    rc = lib.bf1_attn_fwd_noalloc(fake, fake, fake, fake, 1, n, n, 16, 2, 128, 0.0, ctypes.byref(cfg), fake, fake,
                                   None, None)
     assert rc == -2 and b"group" in lib.bf1_last_error()
     rc = lib.bf1_attn_fwd_noalloc(None, fake, fake, fake, 1, 64, 64, 16, 8, 128, 0.0, ctypes.byref(cfg), fake, fake,
