@@ -371,8 +371,9 @@ def topology_sweep(bf1, dev):
 
 def backward_sweep(bf1, dev):
     """Backward over the same route (Section 4.2's gradient gate), one layer, 4K .. 32K: CUDA-event median of
-    10 calls (the call clears and rounds its fp32 dK/dV buffers: included).  FLOPs = 10 * d * pairs * Hq
-    (five MMA groups per block pair against the forward's two)."""
+    10 calls (each derives the inverse route, then runs the dQ and the dK/dV kernel).  FLOPs credited =
+    10 * d * pairs * Hq: the five products of the chain rule per block pair against the forward's two (the
+    two kernels both recompute S and dP, seven MMA groups in all: not credited)."""
     out = []
     stream = torch.cuda.current_stream()
     for name in ("qwen_4k", "qwen_8k", "qwen_16k", "qwen_32k"):
@@ -383,8 +384,7 @@ def backward_sweep(bf1, dev):
         cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
         route = bf1.plan_route(cu, w.max_seqlen)
         o, lse = bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route)
-        ws = torch.empty(int(bf1.load().bf1_attn_bwd_workspace_bytes(w.total_tokens, w.hkv, w.d)), dtype=torch.uint8,
-                         device=dev)
+        ws = bf1.bwd_workspace(route, w.total_tokens, w.hq, w.hkv, w.d, dev)
         f = lambda: bf1.attn_bwd(q, k, v, o, lse, d_o, cu, w.max_seqlen, route, workspace=ws)
         for _ in range(3):
             f()
@@ -506,8 +506,7 @@ def run_single(args):
         d_o = torch.randn(q.shape, generator=torch.Generator(device=dev).manual_seed(w.seed), device=dev,
                           dtype=torch.float32).to(torch.bfloat16)
         bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route, out=o, lse=lse)
-        ws = torch.empty(int(bf1.load().bf1_attn_bwd_workspace_bytes(w.total_tokens, w.hkv, w.d)), dtype=torch.uint8,
-                         device=dev)
+        ws = bf1.bwd_workspace(route, w.total_tokens, w.hq, w.hkv, w.d, dev)
         f = lambda: bf1.attn_bwd(q, k, v, o, lse, d_o, cu, w.max_seqlen, route, workspace=ws)
         pairs = int(2.5 * sum(selected_pairs(n) for n in w.seqlens))   # five MMA groups against the forward's two
     elif args.mode == "dense":

@@ -220,11 +220,16 @@ int bf1_decode_fwd(const void *q, const void *k_pages, const void *v_pages, int3
  * Q, K and V gradients) ---------------------------------------------------------------------------
  * Given the forward's inputs, its outputs o and lse, and the upstream gradient d_o [T, hq, d] bf16,
  * writes dq [T, hq, d], dk and dv [T, hkv, d] in bf16 (the gradients of the G query heads of a KV
- * head add up in dk, dv).  P is recomputed as exp(scale * <q, k> - lse); dk and dv are accumulated
- * in fp32 in `workspace` (bf1_attn_bwd_workspace_bytes() bytes, 16-byte aligned; it is cleared by
- * the call) with floating-point atomics, so their last bits depend on the order of arrival.
- * Head dimension 128 only; other limits as bf1_attn_fwd.  `route` must be the forward's. */
-int64_t bf1_attn_bwd_workspace_bytes(int64_t total_tokens, int32_t hkv, int32_t d);
+ * head add up in dk, dv).  P is recomputed as exp(scale * <q, k> - lse).  dq is computed along the
+ * route (one query block at a time over its list), dk and dv along the inverse route (one KV block
+ * at a time over the query blocks that read it), which the call derives from the lists itself: no
+ * floating-point atomics anywhere, so all three gradients come out bit-identical on every run.
+ * `workspace` (bf1_attn_bwd_workspace_bytes() bytes, 256-byte aligned, contents irrelevant on entry)
+ * holds the row terms <d_o, o>, the inverse route and the partial sums of KV blocks with very many
+ * readers.  Geometry limits as bf1_attn_fwd.  `route` must be the forward's (host struct; only its
+ * capacities are used by the size helper). */
+int64_t bf1_attn_bwd_workspace_bytes(const bf1_route *route /* host */, int64_t total_tokens,
+                                     int32_t hq, int32_t hkv, int32_t d);
 int bf1_attn_bwd(const void *q, const void *k, const void *v, const void *o, const float *lse,
                  const void *d_o, const int32_t *cu_seqlens_dev, int32_t batch, int64_t total_tokens,
                  int32_t max_seqlen, int32_t hq, int32_t hkv, int32_t d, float softmax_scale,

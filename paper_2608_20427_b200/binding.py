@@ -85,7 +85,7 @@ def load():
     L.bf1_decode_fwd.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, f32, ctypes.POINTER(_DecodePlanC), vp, vp,
                                  vp, vp]
     L.bf1_attn_bwd_workspace_bytes.restype = i64
-    L.bf1_attn_bwd_workspace_bytes.argtypes = [i64, i32, i32]
+    L.bf1_attn_bwd_workspace_bytes.argtypes = [ctypes.POINTER(_RouteC), i64, i32, i32, i32]
     L.bf1_attn_bwd.restype = ctypes.c_int
     L.bf1_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, f32, ctypes.POINTER(_RouteC),
                                vp, vp, vp, vp, vp]
@@ -308,14 +308,19 @@ def decode_fwd(q, k_pages, v_pages, seqlens, plan: DecodePlan, workspace, scale:
     return out, lse
 
 
+def bwd_workspace(route: Route, total_tokens: int, hq: int, hkv: int, d: int, device) -> torch.Tensor:
+    """Scratch for attn_bwd (reusable; its contents do not matter on entry)."""
+    nbytes = int(load().bf1_attn_bwd_workspace_bytes(ctypes.byref(route.c), total_tokens, hq, hkv, d))
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
 def attn_bwd(q, k, v, o, lse, d_o, cu_seqlens, max_seqlen: int, route: Route, scale: Optional[float] = None,
              workspace=None, stream=None):
     """bf1_attn_bwd: (dq, dk, dv) in bf16 for the upstream gradient d_o; d = 128 only."""
     T, hq, hkv, d = _check_qkv(q, k, v)
     assert d_o.shape == q.shape and d_o.dtype == torch.bfloat16 and d_o.is_contiguous()
     if workspace is None:
-        workspace = torch.empty(max(int(load().bf1_attn_bwd_workspace_bytes(T, hkv, d)), 16), dtype=torch.uint8,
-                                device=q.device)
+        workspace = bwd_workspace(route, T, hq, hkv, d, q.device)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
     _check(load().bf1_attn_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
                                cu_seqlens.data_ptr(), cu_seqlens.numel() - 1, T, max_seqlen, hq, hkv, d,

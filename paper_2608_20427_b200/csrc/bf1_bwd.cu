@@ -4,22 +4,31 @@
 // The paper's correctness gates include a backward pass with finite Q, K and V gradients (Section
 // 4.2).  With P = exp(S - LSE) recomputed from the saved LSE and D_i = <dO_i, O_i>:
 //     dV_p += P^T dO,   dP = dO V_p^T,   dS = P o (dP - D) * scale,   dQ += dS K_p,   dK_p += dS^T Q.
-// Work unit = (query block, KV head) as in the forward pass: the two grouped query heads are the
-// 128 rows of every MMA, so their contributions to dK / dV add up inside the tensor core.  Per
-// list entry p, five groups of tcgen05 MMAs:
-//     S    = Q   K_p^T        (128 x 64 x 128)   A, B K-major from shared memory
-//     dP   = dO  V_p^T        (128 x 64 x 128)   same layouts
-//     dQ  += dS  K_p          (128 x 128 x 64)   A = dS (bf16, written to shared memory by the threads,
-//                                                K-major), B = K_p MN-major; accumulates in TMEM
-//     dV^T = dO^T P           (128 x 64 x 128)   A = dO MN-major, B = P MN-major (row-major [q][kv] tile)
-//     dK^T = Q^T  dS          (128 x 64 x 128)   A = Q MN-major,  B = dS MN-major
-// dV^T / dK^T come out with the head dimension on the TMEM lanes; each thread adds its 64 values
-// into fp32 accumulation buffers with coalesced red.global.add.f32 (several query blocks read the
-// same KV block), and a second kernel rounds those buffers to bf16.  One CTA per unit and pair of
-// query heads (G = 4: two CTAs per unit, whose dK / dV contributions meet in the fp32 buffers; G = 1:
-// the second head's rows are cleared and contribute nothing), single-buffered, every step in sequence.
-// With d = 64 the transposed products still run as M = 128 MMAs: tensor-memory lanes 64..127 then hold
-// nothing of value and are not read.
+// dQ of a query block sums over the KV blocks of its list; dK / dV of a KV block sum over the query
+// blocks that read it.  So there are two kernels, each walking the route in the direction in which its
+// output stays put, and nothing is ever added in global memory (no atomics, no fp32 gradient buffers,
+// the same bits on every run):
+//
+//   bwd_dq_kernel    unit = (query block, KV head, pair of query heads), as in the forward pass: the two
+//                    heads are the 128 rows of every MMA.  Per list entry p:
+//                        S  = Q  K_p^T   (128 x 64 x d)    A, B K-major from shared memory
+//                        dP = dO V_p^T   (128 x 64 x d)
+//                        dQ += dS K_p    (128 x d x 64)    A = dS (bf16, written to shared memory by the
+//                                                          threads), B = K_p MN-major; accumulates in TMEM
+//                    It also leaves D_i in the workspace for the second kernel.
+//   bwd_dkv_kernel   unit = (KV block p, KV head, a run of the query blocks that read p): the INVERSE
+//                    route, which three small kernels derive from the lists on every call (any lists: the
+//                    planner's or the caller's).  Per reader j (and pair of heads), S and dP as above, then
+//                        dV^T += dO^T P  (d x 64 x 128)    A = dO MN-major, B = P MN-major ([q][kv] tile)
+//                        dK^T += Q^T  dS (d x 64 x 128)    A = Q MN-major,  B = dS MN-major
+//                    accumulating in tensor memory across all readers (head dimension on the lanes), and
+//                    one store at the end.  A block with very many readers (block 0: every query block)
+//                    is cut into runs of `chunk` readers handled by different CTAs; their fp32 partial
+//                    sums are added in run order by bwd_combine_kernel.
+//
+// Both compute kernels are one CTA per unit, two CTAs per SM, every step of a tile in sequence; P is
+// rounded to bf16 before the MMAs, as in the forward.  With d = 64 the transposed products still run as
+// M = 128 MMAs: tensor-memory lanes 64..127 then hold nothing of value and are not read.
 #include <cuda.h>
 
 #include "bf1_common.cuh"
@@ -28,6 +37,23 @@ namespace bf1 {
 
 constexpr int kBlock64 = 64;     // b: tokens per block
 constexpr int kBwdThreads = 128;
+constexpr int kMinChunk = 16;    // readers per dK/dV unit, at least
+
+// The inverse route and the units of bwd_dkv_kernel, all inside the caller's workspace.
+struct InvPlan {
+    int32_t* count;       // [cap] readers of KV slot g (with multiplicity)
+    int32_t* start;       // [cap + 1] first reader of slot g in `readers`
+    int32_t* chunks;      // [cap] runs the slot's readers are cut into
+    int32_t* part0;       // [cap] first partial-sum slot of a slot with more than one run, else -1
+    int32_t* wofs;        // [cap * 8] where each of the eight scanning warps writes inside the slot's readers
+    int32_t* readers;     // [cap * max_degree] query slots, ascending per KV slot
+    int32_t* unit_slot;   // [max_units] KV slot of the unit
+    int32_t* unit_begin;  // [max_units] its readers: readers[begin .. end)
+    int32_t* unit_end;
+    int32_t* unit_part;   // [max_units] partial-sum slot it writes, or -1: it writes the final bf16 rows
+    int32_t* scalars;     // [4] number of units, total readers, chunk, partial slots
+    int32_t cap, max_units;
+};
 
 struct BwdArgs {
     const int32_t* cu_seqlens;
@@ -42,10 +68,21 @@ struct BwdArgs {
     const __nv_bfloat16* o;
     const __nv_bfloat16* d_o;
     const float* lse;
+    float* delta;          // [hq, T] D_i = <dO_i, O_i>: written by the dQ kernel, read by the dK/dV kernel
     __nv_bfloat16* dq;
-    float* dk32;   // [T, hkv, d] fp32 accumulation
-    float* dv32;
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    float* partial;        // [partial slots][hkv][2][64][d] fp32 sums of the runs of a many-reader block
+    InvPlan inv;
 };
+
+// Entry e of a list as every kernel of this library uses it: kept inside [0, j], the last entry the
+// query block itself, whatever the array holds (a caller's route may be wrong; the forward flags it).
+__device__ __forceinline__ int list_entry(const int32_t* list, int e, int cnt, int j) {
+    int p = list[e];
+    if (p < 0 || p > j || (e == cnt - 1) != (p == j)) p = (e == cnt - 1) ? j : 0;
+    return p;
+}
 
 template <int D>
 struct BwdSmem {
@@ -55,25 +92,122 @@ struct BwdSmem {
     static constexpr int kDO = kQ + kQBytes;
     static constexpr int kK = kDO + kQBytes;
     static constexpr int kV = kK + kKVBytes;
-    // P [128 q rows][64 kv] bf16, 128-byte rows, swizzled (16 KB).  At d = 128 it takes over V's buffer once
-    // dP = dO V^T has been computed; at d = 64 the V tile is only 8 KB, so P gets room of its own.
-    static constexpr int kP = D == 128 ? kV : kV + kKVBytes;
-    static constexpr int kDS = kP + 16384;           // dS same layout
-    static constexpr int kBar = kDS + 16384;
-    static constexpr int kTotal = kBar + 64;
+    // P and dS: [128 q rows][64 kv] bf16, 128-byte rows, swizzled (16 KB each).
+    //   dQ kernel:    only dS is needed; it has room of its own.
+    //   dK/dV kernel: at d = 128, P takes over V's buffer and dS takes over K's once S and dP have been
+    //                 computed (K and V are fetched again for the next reader; they come from L2); at d = 64 the
+    //                 K / V tiles are only 8 KB, so P and dS get room of their own.
+    static constexpr int kDS_dq = kV + kKVBytes;
+    static constexpr int kBar_dq = kDS_dq + 16384;
+    static constexpr int kTotal_dq = kBar_dq + 64;
+    static constexpr int kP_kv = D == 128 ? kV : kV + kKVBytes;
+    static constexpr int kDS_kv = D == 128 ? kK : kP_kv + 16384;
+    static constexpr int kBar_kv = D == 128 ? kV + kKVBytes : kDS_kv + 16384;
+    static constexpr int kTotal_kv = kBar_kv + 64;
 };
 
+// ---- pieces shared by the two compute kernels ------------------------------------------------------------------
+
+// S = Q K^T and dP = dO V^T: D / 16 k-steps over the head dimension (thread 0 only).
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q,
-                                                               const __grid_constant__ CUtensorMap tm_k,
-                                                               const __grid_constant__ CUtensorMap tm_v,
-                                                               const __grid_constant__ CUtensorMap tm_do,
-                                                               const BwdArgs a) {
+__device__ __forceinline__ void issue_s_dp(uint32_t t_s, uint32_t t_dp, uint32_t sQ, uint32_t sDO, uint32_t sK, uint32_t sV) {
+    constexpr uint32_t kHi = desc_hi_sw128(1024);
+    constexpr uint32_t kIdS = idesc_bf16_f32_ab(64, false, false);     // 128 x 64, A and B K-major
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
+        if (kk == 0) {
+            mma_ss_lohi<false>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
+            mma_ss_lohi<false>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
+        } else {
+            mma_ss_lohi<true>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
+            mma_ss_lohi<true>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
+        }
+    }
+}
+
+// P and dS of this thread's row from S and dP in tensor memory, written as bf16 rows (128-byte rows, 16-byte
+// chunks XOR-swizzled with the row) where the next MMAs read them.  Masked entries get s = -inf (self block,
+// warp-uniform branch) and rows outside the sequence an infinite LSE: both give P = 0 exactly, and with it dS = 0.
+template <bool kWriteP>
+__device__ __forceinline__ void p_and_ds(uint32_t t_s, uint32_t t_dp, uint32_t prow, uint32_t dsrow, int tid, int tl, bool diag,
+                                         float lse_row2, float drow, float scale, float scale_log2) {
+    const uint64_t c2p = pack2(scale_log2, scale_log2), nlp = pack2(-lse_row2, -lse_row2);
+    const uint64_t scp = pack2(scale, scale), ndp = pack2(-drow * scale, -drow * scale);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint32_t sr[32], dr[32];
+        tmem_ld32(t_s + half * 32, sr);
+        tmem_ld32(t_dp + half * 32, dr);
+        tmem_wait_ld();
+        if (diag) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+                if (half * 32 + c > tl) sr[c] = 0xff800000u;   // -inf: causal triangle
+        }
+        uint32_t pw[16], dw[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            const uint64_t x = fma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), c2p, nlp);
+            float x0, x1;
+            unpack2(x, x0, x1);
+            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+            // dS = P * (dP - D) * scale
+            const uint64_t t = fma2(pack2(__uint_as_float(dr[2 * c]), __uint_as_float(dr[2 * c + 1])), scp, ndp);
+            float d0, d1;
+            unpack2(mul2(pack2(p0, p1), t), d0, d1);
+            pw[c] = pack_bf16x2(p0, p1);
+            dw[c] = pack_bf16x2(d0, d1);
+        }
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk half * 4 + c4 of the 128-byte row
+            const int ch = (half * 4 + c4) ^ (tid & 7);
+            if (kWriteP) st_shared_v4(prow + (ch << 4), pw[4 * c4], pw[4 * c4 + 1], pw[4 * c4 + 2], pw[4 * c4 + 3]);
+            st_shared_v4(dsrow + (ch << 4), dw[4 * c4], dw[4 * c4 + 1], dw[4 * c4 + 2], dw[4 * c4 + 3]);
+        }
+    }
+}
+
+// One head per KV head: rows 64..127 of every column chunk of the Q and dO tiles are never written by a copy;
+// the MMAs still read them, so they are cleared once (they then give P = 0 and dS = 0 like rows past a sequence).
+template <int D>
+__device__ __forceinline__ void clear_idle_rows(uint32_t sQ, uint32_t sDO, int tid) {
+    for (int i = tid; i < 2 * (D / 64) * 512; i += kBwdThreads) {
+        const int which = i / ((D / 64) * 512), ch = (i / 512) % (D / 64), off = i % 512;
+        st_shared_v4((which ? sDO : sQ) + ch * 16384 + 8192 + off * 16, 0u, 0u, 0u, 0u);
+    }
+    fence_proxy_async();
+}
+
+// Q and dO tiles of one query block and pair of heads (thread 0 only; expect_tx is the caller's).
+template <int D>
+__device__ __forceinline__ void load_q_do(uint32_t sQ, uint32_t sDO, const CUtensorMap* tm_q, const CUtensorMap* tm_do, int tok0,
+                                          int head, int group, uint32_t bar) {
+    if (group > 1) {
+        tma_load_4d(sQ, tm_q, 0, tok0, head, 0, bar);
+        tma_load_4d(sDO, tm_do, 0, tok0, head, 0, bar);
+    } else {
+#pragma unroll
+        for (int ch = 0; ch < D / 64; ++ch) {
+            tma_load_4d(sQ + ch * 16384, tm_q, 0, tok0, head, ch, bar);
+            tma_load_4d(sDO + ch * 16384, tm_do, 0, tok0, head, ch, bar);
+        }
+    }
+}
+
+// ---- dQ --------------------------------------------------------------------------------------------------------
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                             const __grid_constant__ CUtensorMap tm_k,
+                                                             const __grid_constant__ CUtensorMap tm_v,
+                                                             const __grid_constant__ CUtensorMap tm_do,
+                                                             const BwdArgs a) {
     using L = BwdSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     // no static shared memory: it would cost a whole extra kilobyte and with it the second CTA per SM
-    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar + 32);
-    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar + 36);
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_dq + 40);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_dq + 44);
     const int tid = threadIdx.x, warp = tid >> 5;
     const int slot = blockIdx.x, kvh = blockIdx.y, pair = blockIdx.z;   // pair: which two query heads of the group
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
@@ -87,14 +221,14 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
     const int tok0 = seq0 + j * kBlock64;
 
     const uint32_t base = smem_u32(smem);
-    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV;
-    const uint32_t sP = base + L::kP, sDS = base + L::kDS;
-    const uint32_t bar_q = base + L::kBar, bar_kv = bar_q + 8, bar_a = bar_q + 16, bar_b = bar_q + 24;
+    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV, sDS = base + L::kDS_dq;
+    const uint32_t bar_q = base + L::kBar_dq, bar_k = bar_q + 8, bar_v = bar_q + 16, bar_a = bar_q + 24, bar_b = bar_q + 32;
     if (tid == 0) {
         s_abort = (base & 1023u) ? 1 : 0;
         if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
         mbar_init(bar_q, 1);
-        mbar_init(bar_kv, 1);
+        mbar_init(bar_k, 1);
+        mbar_init(bar_v, 1);
         mbar_init(bar_a, 1);
         mbar_init(bar_b, 1);
         fence_mbar_init();
@@ -104,14 +238,13 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
         tmem_alloc(smem_u32(&s_tmem), 256);
         tmem_relinquish();
     }
+    if (a.group == 1) clear_idle_rows<D>(sQ, sDO, tid);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* abort_flag = &s_abort;
-    // dV^T and dK^T reuse the columns of S and dP (which the threads have turned into P and dS by then):
-    // 256 columns and 112 KB of shared memory per CTA let two CTAs share an SM
-    constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128, kColDVt = kColS, kColDKt = kColDP;
+    constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128;
     const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
 
     // rows of this thread: head hl, token tl of the query block
@@ -120,32 +253,24 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
     const int tok = tok0 + tl;
     const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;   // G = 1: rows 64..127 belong to no head
 
-    if (a.group == 1) {
-        // one head: rows 64..127 of every column chunk of the Q and dO tiles are never written by a copy; the
-        // MMAs still read them, so they are cleared (they then give P = 0 and dS = 0 like rows past a sequence)
-        for (int i = tid; i < 2 * (D / 64) * 512; i += kBwdThreads) {
-            const int which = i / ((D / 64) * 512), ch = (i / 512) % (D / 64), off = i % 512;
-            st_shared_v4((which ? sDO : sQ) + ch * 16384 + 8192 + off * 16, 0u, 0u, 0u, 0u);
-        }
-        fence_proxy_async();
-        __syncthreads();
-    }
+    // K and V have a barrier each: V is free as soon as dP has been computed, K only after dQ += dS K
+    auto load_k = [&](int p) {   // thread 0 only
+        mbar_expect_tx(bar_k, L::kKVBytes);
+        tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_k);
+    };
+    auto load_v = [&](int p) {
+        mbar_expect_tx(bar_v, L::kKVBytes);
+        tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_v);
+    };
     if (tid == 0 && !s_abort) {
-        if (a.group > 1) {
-            mbar_expect_tx(bar_q, 2 * L::kQBytes);
-            tma_load_4d(sQ, &tm_q, 0, tok0, h, 0, bar_q);      // h: the pair's first head (hl = 0 here)
-            tma_load_4d(sDO, &tm_do, 0, tok0, h, 0, bar_q);
-        } else {
-            mbar_expect_tx(bar_q, L::kQBytes);                 // 64 rows of each
-#pragma unroll
-            for (int ch = 0; ch < D / 64; ++ch) {
-                tma_load_4d(sQ + ch * 16384, &tm_q, 0, tok0, h, ch, bar_q);
-                tma_load_4d(sDO + ch * 16384, &tm_do, 0, tok0, h, ch, bar_q);
-            }
-        }
+        mbar_expect_tx(bar_q, a.group > 1 ? 2 * L::kQBytes : L::kQBytes);
+        load_q_do<D>(sQ, sDO, &tm_q, &tm_do, tok0, kvh * a.group + pair * 2, a.group, bar_q);
+        const int p0 = list_entry(list, 0, cnt, j);
+        load_k(p0);
+        load_v(p0);
     }
     // D_i = <dO_i, O_i> and the row's LSE in the log2 domain
-    float Drow = 0.f, lse2 = 0.f;
+    float Drow = 0.f, lse2 = INFINITY;
     if (row_ok) {
         const uint4* op = reinterpret_cast<const uint4*>(a.o + ((size_t)tok * a.hq + h) * D);
         const uint4* gp = reinterpret_cast<const uint4*>(a.d_o + ((size_t)tok * a.hq + h) * D);
@@ -160,94 +285,27 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
             }
         }
         lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
+        a.delta[(size_t)h * a.total_tokens + tok] = Drow;   // for the dK/dV kernel
     }
     mbar_wait(bar_q, 0, abort_flag, a.status);
 
     constexpr uint32_t kHi = desc_hi_sw128(1024);
-    constexpr uint32_t kIdS = idesc_bf16_f32_ab(64, false, false);     // S, dP: 128 x 64, A and B K-major
-    constexpr uint32_t kIdQ = idesc_bf16_f32_ab(D, false, true);       // dQ: 128 x 128, B (K tile) MN-major
-    constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);       // dV^T, dK^T: A and B MN-major
-
-    // list entry -> block index, kept inside the sequence whatever the list holds
-    auto entry = [&](int it) -> int {
-        int p = list[it];
-        if (p < 0 || p > j || (it == cnt - 1) != (p == j)) {
-            if (tid == 0 && a.status) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
-            p = (it == cnt - 1) ? j : 0;
-        }
-        return p;
-    };
-    auto load_kv = [&](int p) {   // thread 0 only
-        mbar_expect_tx(bar_kv, 2 * L::kKVBytes);
-        tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
-        tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_kv);
-    };
-    int p = entry(0);
-    if (tid == 0) load_kv(p);
+    constexpr uint32_t kIdQ = idesc_bf16_f32_ab(D, false, true);       // dQ: 128 x d, B (K tile) MN-major
     for (int it = 0; it < cnt; ++it) {
-        const int p_next = (it + 1 < cnt) ? entry(it + 1) : 0;
+        const int p_next = (it + 1 < cnt) ? list_entry(list, it + 1, cnt, j) : 0;
         const bool diag = (it == cnt - 1);
-        const int kv_valid = min(kBlock64, seqlen - p * kBlock64);      // key rows of this block inside the sequence
         if (tid == 0) {
-            mbar_wait(bar_kv, it & 1, abort_flag, a.status);
+            mbar_wait(bar_k, it & 1, abort_flag, a.status);
+            mbar_wait(bar_v, it & 1, abort_flag, a.status);
             tc_fence_after();
-            // S = Q K^T and dP = dO V^T: 8 k-steps of 16 over d
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
-                if (kk == 0) {
-                    mma_ss_lohi<false>(tmem + kColS, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
-                    mma_ss_lohi<false>(tmem + kColDP, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
-                } else {
-                    mma_ss_lohi<true>(tmem + kColS, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
-                    mma_ss_lohi<true>(tmem + kColDP, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
-                }
-            }
+            issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sK, sV);
             mma_commit(bar_a);
         }
         __syncwarp();
         mbar_wait(bar_a, it & 1, abort_flag, a.status);
         tc_fence_after();
-
-        // ---- P and dS for this thread's row, 32 columns at a time, written as bf16 rows ------------
-        const uint32_t prow = sP + tid * 128, dsrow = sDS + tid * 128;
-        // masked entries get s = -inf (self block, warp-uniform branch) and rows past the end of the
-        // sequence an infinite LSE: both give P = 0 exactly, and with it dS = 0
-        const float lse_row = row_ok ? lse2 : INFINITY;
-        const uint64_t c2p = pack2(a.scale_log2, a.scale_log2), nlp = pack2(-lse_row, -lse_row);
-        const uint64_t scp = pack2(a.scale, a.scale), ndp = pack2(-Drow * a.scale, -Drow * a.scale);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t sr[32], dr[32];
-            tmem_ld32(t_lane + kColS + half * 32, sr);
-            tmem_ld32(t_lane + kColDP + half * 32, dr);
-            tmem_wait_ld();
-            if (diag) {
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                    if (half * 32 + c > tl) sr[c] = 0xff800000u;   // -inf: causal triangle
-            }
-            uint32_t pw[16], dw[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const uint64_t x = fma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), c2p, nlp);
-                float x0, x1;
-                unpack2(x, x0, x1);
-                const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                // dS = P * (dP - D) * scale
-                const uint64_t t = fma2(pack2(__uint_as_float(dr[2 * c]), __uint_as_float(dr[2 * c + 1])), scp, ndp);
-                float d0, d1;
-                unpack2(mul2(pack2(p0, p1), t), d0, d1);
-                pw[c] = pack_bf16x2(p0, p1);
-                dw[c] = pack_bf16x2(d0, d1);
-            }
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk half * 4 + c4 of the 128-byte row
-                const int ch = (half * 4 + c4) ^ (tid & 7);
-                st_shared_v4(prow + (ch << 4), pw[4 * c4], pw[4 * c4 + 1], pw[4 * c4 + 2], pw[4 * c4 + 3]);
-                st_shared_v4(dsrow + (ch << 4), dw[4 * c4], dw[4 * c4 + 1], dw[4 * c4 + 2], dw[4 * c4 + 3]);
-            }
-        }
+        if (tid == 0 && it + 1 < cnt) load_v(p_next);   // V is free: its next tile travels during the arithmetic below
+        p_and_ds<false>(t_lane + kColS, t_lane + kColDP, 0u, sDS + tid * 128, tid, tl, diag, lse2, Drow, a.scale, a.scale_log2);
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
@@ -263,54 +321,15 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
                 if (it == 0 && kk == 0) mma_ss_lohi<false>(tmem + kColDQ, alo, blo, kHi, kIdQ);
                 else mma_ss_lohi<true>(tmem + kColDQ, alo, blo, kHi, kIdQ);
             }
-            // dV^T = dO^T P and dK^T = Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
-            // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t ko = (kk * 2048) >> 4;
-                if (kk == 0) {
-                    mma_ss_lohi<false>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                    mma_ss_lohi<false>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
-                } else {
-                    mma_ss_lohi<true>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                    mma_ss_lohi<true>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
-                }
-            }
             mma_commit(bar_b);
         }
         __syncwarp();
-        mbar_wait(bar_b, it & 1, abort_flag, a.status);
+        mbar_wait(bar_b, it & 1, abort_flag, a.status);   // K, the dS buffer and the S / dP columns are free again
         tc_fence_after();
-        // K, V (and P, which lives in V's buffer) are free: fetch the next tile while the sums go out
-        if (tid == 0 && it + 1 < cnt) load_kv(p_next);
-
-        // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns -----------------
-        float* dvp = a.dv32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
-        float* dkp = a.dk32 + ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
-        const size_t rstride = (size_t)a.hkv * D;
-        const bool lane_ok = tid < D;   // d = 64: lanes 64..127 of the transposed products hold nothing (warp-uniform)
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t vr[32], kr[32];
-            tmem_ld32(t_lane + kColDVt + half * 32, vr);
-            tmem_ld32(t_lane + kColDKt + half * 32, kr);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const int kvr = half * 32 + c;
-                if (kvr < kv_valid && lane_ok) {
-                    atomicAdd(dvp + kvr * rstride, __uint_as_float(vr[c]));
-                    atomicAdd(dkp + kvr * rstride, __uint_as_float(kr[c]));
-                }
-            }
-        }
-        tc_fence_before();
-        __syncthreads();   // dS buffer and the S/dP/dV^T/dK^T columns are free again
-        p = p_next;
+        if (tid == 0 && it + 1 < cnt) load_k(p_next);
     }
 
     // ---- dQ rows -----------------------------------------------------------------------------------
-    tc_fence_after();
     __nv_bfloat16* dqrow = a.dq + ((size_t)tok * a.hq + h) * D;
 #pragma unroll
     for (int c = 0; c < D / 32; ++c) {
@@ -334,24 +353,346 @@ __global__ void __launch_bounds__(kBwdThreads, 2) attn_bwd_kernel(const __grid_c
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
-// fp32 accumulation buffers -> bf16 gradients
-__global__ void bwd_round_kernel(const float* __restrict__ src_k, const float* __restrict__ src_v,
-                                 __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, size_t n) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        dk[i] = __float2bfloat16_rn(src_k[i]);
-        dv[i] = __float2bfloat16_rn(src_v[i]);
+// ---- the inverse route -----------------------------------------------------------------------------------------
+
+// One CTA per KV slot: its readers are the query slots g >= it of the same sequence whose list names its block
+// (with multiplicity, should a caller's list name a block twice).  The candidates' lists are scanned as one flat
+// array (coalesced), each of the eight warps taking a contiguous eighth of the candidates.  kFill = false counts
+// (per warp, so that the second pass knows where each warp writes), kFill = true writes the readers in ascending
+// order.
+template <bool kFill>
+__global__ void __launch_bounds__(256) inverse_route_kernel(const BwdArgs a) {
+    __shared__ int32_t s_cnt[8];
+    const int gp = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nqb = min(*a.num_qblocks, a.capacity);
+    if (gp >= nqb) return;
+    const int seq = a.qb_seq[gp], p = a.qb_block[gp];
+    const int nb = (a.cu_seqlens[seq + 1] - a.cu_seqlens[seq] + kBlock64 - 1) / kBlock64;
+    const int g_end = min(gp - p + nb, nqb);                 // one past the sequence's last query slot
+    const int span = (g_end - gp + 7) / 8;
+    const int g_lo = min(gp + warp * span, g_end), g_hi = min(g_lo + span, g_end);
+    const int flat = (g_hi - g_lo) * a.max_degree;           // this warp's part of the flat (slot, entry) array
+    int total = 0;
+    int32_t* out = kFill ? a.inv.readers + a.inv.start[gp] + a.inv.wofs[gp * 8 + warp] : nullptr;
+    for (int f0 = 0; f0 < flat; f0 += 32) {
+        const int f = f0 + lane;
+        bool match = false;
+        int g = 0;
+        if (f < flat) {
+            g = g_lo + f / a.max_degree;
+            const int e = f % a.max_degree;
+            const int cnt = min(max(a.kv_count[g], 1), a.max_degree);
+            if (e < cnt) match = list_entry(a.kv_idx + (size_t)g * a.max_degree, e, cnt, a.qb_block[g]) == p;
+        }
+        const unsigned hits = __ballot_sync(0xffffffffu, match);
+        if (kFill && match) out[total + __popc(hits & ((1u << lane) - 1))] = g;
+        total += __popc(hits);
+    }
+    if (!kFill) {
+        if (lane == 0) s_cnt[warp] = total;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int run = 0;
+            for (int w = 0; w < 8; ++w) {
+                a.inv.wofs[gp * 8 + w] = run;
+                run += s_cnt[w];
+            }
+            a.inv.count[gp] = run;
+        }
+    }
+}
+
+// One CTA: offsets of the reader lists, the run length, and the units of the dK/dV kernel.
+__global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a) {
+    __shared__ int32_t s_warp[32];
+    __shared__ int32_t s_carry[3];
+    __shared__ int32_t s_chunk;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nqb = min(*a.num_qblocks, a.capacity);
+    const InvPlan& v = a.inv;
+    // exclusive scan of x over the CTA, with a running carry in s_carry[which]
+    auto scan = [&](int x, int which, int& excl) {
+        int incl = x;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int w = s_warp[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, w, off);
+                if (lane >= off) w += up;
+            }
+            s_warp[lane] = w;
+        }
+        __syncthreads();
+        const int before = (warp > 0 ? s_warp[warp - 1] : 0) + s_carry[which];
+        excl = before + incl - x;
+        const int chunk_total = s_warp[31];
+        __syncthreads();
+        if (tid == 0) s_carry[which] += chunk_total;
+        __syncthreads();
+    };
+    if (tid < 3) s_carry[tid] = 0;
+    __syncthreads();
+    // pass 1: where each slot's readers start; the total decides the run length
+    for (int b0 = 0; b0 < nqb; b0 += 1024) {
+        const int g = b0 + tid;
+        const int c = g < nqb ? v.count[g] : 0;
+        int excl;
+        scan(c, 0, excl);
+        if (g < nqb) v.start[g] = excl;
+    }
+    if (tid == 0) {
+        const int total = s_carry[0];
+        v.start[nqb] = total;
+        // runs of at least kMinChunk readers, and long enough that the slots with more than one run cannot need
+        // more than `cap` partial-sum slots between them (such a slot has fewer than 2 * count / chunk runs)
+        s_chunk = max(kMinChunk, (2 * total + max(v.cap, 1) - 1) / max(v.cap, 1));
+    }
+    __syncthreads();
+    const int chunk = s_chunk;
+    // pass 2: runs per slot -> unit numbers and partial-sum slots
+    for (int b0 = 0; b0 < nqb; b0 += 1024) {
+        const int g = b0 + tid;
+        const int c = g < nqb ? v.count[g] : 0;
+        const int runs = (c + chunk - 1) / chunk;
+        int u0, q0;
+        scan(runs, 1, u0);
+        scan(runs > 1 ? runs : 0, 2, q0);
+        if (g < nqb) {
+            v.chunks[g] = runs;
+            v.part0[g] = runs > 1 ? q0 : -1;
+            const int first = v.start[g];
+            for (int r = 0; r < runs; ++r) {
+                if (u0 + r >= v.max_units) break;
+                v.unit_slot[u0 + r] = g;
+                v.unit_begin[u0 + r] = first + r * chunk;
+                v.unit_end[u0 + r] = min(first + c, first + (r + 1) * chunk);
+                v.unit_part[u0 + r] = runs > 1 ? q0 + r : -1;
+            }
+        }
+    }
+    if (tid == 0) {
+        const bool fits = s_carry[1] <= v.max_units && s_carry[2] <= v.cap;
+        if (!fits && a.status) atomicOr(a.status, BF1_DEV_CAPACITY);
+        v.scalars[0] = fits ? s_carry[1] : 0;
+        v.scalars[1] = s_carry[0];
+        v.scalars[2] = chunk;
+        v.scalars[3] = s_carry[2];
+    }
+}
+
+// ---- dK, dV ----------------------------------------------------------------------------------------------------
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                              const __grid_constant__ CUtensorMap tm_k,
+                                                              const __grid_constant__ CUtensorMap tm_v,
+                                                              const __grid_constant__ CUtensorMap tm_do,
+                                                              const BwdArgs a) {
+    using L = BwdSmem<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_kv + 32);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_kv + 36);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int unit = blockIdx.x, kvh = blockIdx.y;
+    if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
+    if (unit >= a.inv.scalars[0]) return;
+    const int gp = a.inv.unit_slot[unit];
+    const int r_begin = a.inv.unit_begin[unit], r_end = a.inv.unit_end[unit], part = a.inv.unit_part[unit];
+    const int seq = a.qb_seq[gp], p = a.qb_block[gp];
+    const int seq0 = a.cu_seqlens[seq];
+    const int seqlen = a.cu_seqlens[seq + 1] - seq0;
+    const int kv_valid = min(kBlock64, seqlen - p * kBlock64);      // key rows of this block inside the sequence
+    const int pairs = a.group == 4 ? 2 : 1;
+
+    const uint32_t base = smem_u32(smem);
+    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV;
+    const uint32_t sP = base + L::kP_kv, sDS = base + L::kDS_kv;
+    const uint32_t bar_ld = base + L::kBar_kv, bar_a = bar_ld + 8, bar_b = bar_ld + 16;
+    if (tid == 0) {
+        s_abort = (base & 1023u) ? 1 : 0;
+        if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
+        mbar_init(bar_ld, 1);
+        mbar_init(bar_a, 1);
+        mbar_init(bar_b, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&s_tmem), 256);
+        tmem_relinquish();
+    }
+    if (a.group == 1) clear_idle_rows<D>(sQ, sDO, tid);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    volatile int* abort_flag = &s_abort;
+    // S and dP are recomputed for every reader; dV^T and dK^T stay where they are until the last one
+    constexpr uint32_t kColS = 0, kColDP = 64, kColDVt = 128, kColDKt = 192;
+    const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    const int hl = tid >> 6, tl = tid & 63;
+    constexpr uint32_t kHi = desc_hi_sw128(1024);
+    constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);       // dV^T, dK^T: A and B MN-major
+
+    const int steps = (r_end - r_begin) * pairs;
+    // thread 0 only: Q, dO of query block jq (a block of this block's own sequence) and pair; K, V of this block again
+    auto issue_loads = [&](int jq, int pair) {
+        mbar_expect_tx(bar_ld, (a.group > 1 ? 2 * L::kQBytes : L::kQBytes) + 2 * L::kKVBytes);
+        load_q_do<D>(sQ, sDO, &tm_q, &tm_do, seq0 + jq * kBlock64, kvh * a.group + pair * 2, a.group, bar_ld);
+        tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
+        tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
+    };
+    // the reader of a step and its block index are fetched one step ahead: two dependent global loads that
+    // would otherwise sit in front of every copy
+    int g_next = steps > 0 ? a.inv.readers[r_begin] : gp;
+    int jq_next = a.qb_block[g_next];
+    if (tid == 0 && !s_abort && steps > 0) issue_loads(jq_next, 0);
+    for (int step = 0; step < steps; ++step) {
+        const int g = g_next, jq = jq_next, pair = step % pairs;
+        if (step + 1 < steps) {
+            g_next = a.inv.readers[r_begin + (step + 1) / pairs];
+            jq_next = a.qb_block[g_next];
+        }
+        const int rows_valid = min(kBlock64, seqlen - jq * kBlock64);
+        const int h = kvh * a.group + pair * 2 + hl;
+        const int tok = seq0 + jq * kBlock64 + tl;
+        const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;
+        // the row's LSE (log2 domain) and D_i, fetched while the tiles travel
+        float lse2 = INFINITY, drow = 0.f;
+        if (row_ok) {
+            lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
+            drow = a.delta[(size_t)h * a.total_tokens + tok];
+        }
+        if (tid == 0) {
+            mbar_wait(bar_ld, step & 1, abort_flag, a.status);
+            tc_fence_after();
+            issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sK, sV);
+            mma_commit(bar_a);
+        }
+        __syncwarp();
+        mbar_wait(bar_a, step & 1, abort_flag, a.status);
+        tc_fence_after();
+        p_and_ds<true>(t_lane + kColS, t_lane + kColDP, sP + tid * 128, sDS + tid * 128, tid, tl, g == gp, lse2, drow, a.scale,
+                       a.scale_log2);
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            // dV^T += dO^T P and dK^T += Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
+            // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t ko = (kk * 2048) >> 4;
+                if (kk == 0 && step == 0) {
+                    mma_ss_lohi<false>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                    mma_ss_lohi<false>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                } else {
+                    mma_ss_lohi<true>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                    mma_ss_lohi<true>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                }
+            }
+            mma_commit(bar_b);
+        }
+        __syncwarp();
+        mbar_wait(bar_b, step & 1, abort_flag, a.status);   // every buffer is free again
+        tc_fence_after();
+        if (tid == 0 && step + 1 < steps) issue_loads(jq_next, (step + 1) % pairs);
+    }
+
+    // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns -----------------------
+    if (tid < D && steps > 0) {   // d = 64: lanes 64..127 hold nothing (warp-uniform)
+        const size_t rstride = (size_t)a.hkv * D;
+        const size_t row0 = ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
+        float* pk = part >= 0 ? a.partial + (((size_t)part * a.hkv + kvh) * 2) * (kBlock64 * D) + tid : nullptr;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t vr[32], kr[32];
+            tmem_ld32(t_lane + kColDVt + half * 32, vr);
+            tmem_ld32(t_lane + kColDKt + half * 32, kr);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const int kvr = half * 32 + c;
+                if (kvr < kv_valid) {
+                    if (part < 0) {
+                        a.dv[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(vr[c]));
+                        a.dk[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(kr[c]));
+                    } else {
+                        pk[kvr * D] = __uint_as_float(kr[c]);
+                        pk[kBlock64 * D + kvr * D] = __uint_as_float(vr[c]);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 256);
+}
+
+// KV blocks whose readers were cut into several runs: add the runs' partial sums in run order.
+template <int D>
+__global__ void __launch_bounds__(256) bwd_combine_kernel(const BwdArgs a) {
+    const int gp = blockIdx.x, kvh = blockIdx.y;
+    if (gp >= min(*a.num_qblocks, a.capacity) || a.inv.scalars[0] == 0) return;
+    const int runs = a.inv.chunks[gp], q0 = a.inv.part0[gp];
+    if (runs <= 1) return;
+    const int seq = a.qb_seq[gp], p = a.qb_block[gp];
+    const int seq0 = a.cu_seqlens[seq];
+    const int kv_valid = min(kBlock64, a.cu_seqlens[seq + 1] - seq0 - p * kBlock64);
+    for (int i = threadIdx.x; i < kv_valid * D; i += 256) {
+        float sk = 0.f, sv = 0.f;
+        for (int r = 0; r < runs; ++r) {
+            const float* pk = a.partial + (((size_t)(q0 + r) * a.hkv + kvh) * 2) * (kBlock64 * D);
+            sk += pk[i];
+            sv += pk[kBlock64 * D + i];
+        }
+        const size_t o = ((size_t)(seq0 + p * kBlock64 + i / D) * a.hkv + kvh) * D + i % D;
+        a.dk[o] = __float2bfloat16_rn(sk);
+        a.dv[o] = __float2bfloat16_rn(sv);
     }
 }
 
 int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int heads_per_box, int chunks_per_box);   // bf1_attn.cu
 
+// Where everything lives in the caller's workspace (256-byte aligned sections).
+struct BwdLayout {
+    size_t delta, ints, partial, total;
+    size_t n_count, n_start, n_chunks, n_part0, n_wofs, n_readers, n_units;
+    BwdLayout(int64_t T, int hq, int hkv, int d, int cap, int max_degree) {
+        auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+        n_count = (size_t)cap;
+        n_start = (size_t)cap + 1;
+        n_chunks = (size_t)cap;
+        n_part0 = (size_t)cap;
+        n_wofs = 8 * (size_t)cap;
+        n_readers = (size_t)cap * max_degree;
+        n_units = 2 * (size_t)cap;
+        delta = 0;
+        ints = up((size_t)T * hq * sizeof(float));
+        const size_t n_ints = n_count + n_start + n_chunks + n_part0 + n_wofs + n_readers + 4 * n_units + 4;
+        partial = ints + up(n_ints * sizeof(int32_t));
+        total = partial + up((size_t)cap * hkv * 2 * kBlock64 * d * sizeof(float));
+    }
+};
+
 }  // namespace bf1
 
 using namespace bf1;
 
-extern "C" int64_t bf1_attn_bwd_workspace_bytes(int64_t total_tokens, int32_t hkv, int32_t d) {
-    if (total_tokens < 0 || hkv <= 0 || d <= 0) return -1;
-    return 2 * total_tokens * hkv * d * (int64_t)sizeof(float);
+extern "C" int64_t bf1_attn_bwd_workspace_bytes(const bf1_route* route, int64_t total_tokens, int32_t hq, int32_t hkv,
+                                                int32_t d) {
+    if (!route || total_tokens < 0 || hq <= 0 || hkv <= 0 || d <= 0 || route->capacity_qblocks < 1 || route->max_degree < 1)
+        return -1;
+    return (int64_t)BwdLayout(total_tokens, hq, hkv, d, route->capacity_qblocks, route->max_degree).total;
 }
 
 extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse,
@@ -369,8 +710,9 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
         return fail(BF1_ERR_UNSUPPORTED, "GQA group size %d: only G = 1, 2 and 4 are supported", group);
     if (d != 64 && d != 128) return fail(BF1_ERR_UNSUPPORTED, "head dimension %d: only 64 and 128 are supported", d);
     if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o | (uintptr_t)d_o | (uintptr_t)dq | (uintptr_t)dk |
-         (uintptr_t)dv | (uintptr_t)workspace) & 15)
-        return fail(BF1_ERR_INVALID_ARG, "tensors and workspace must be 16-byte aligned");
+         (uintptr_t)dv) & 15)
+        return fail(BF1_ERR_INVALID_ARG, "tensors must be 16-byte aligned");
+    if ((uintptr_t)workspace & 255) return fail(BF1_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
     if (!route->qb_seq || !route->qb_block || !route->kv_count || !route->kv_idx || !route->num_qblocks || !route->status)
         return fail(BF1_ERR_INVALID_ARG, "a route array pointer is null");
     if (route->capacity_qblocks < 1 || route->max_degree < 1 || hkv > 65535)
@@ -380,13 +722,20 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     BF1_CUDA_CHECK(cudaGetDevice(&dev));
     BF1_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
     if (major != 10) return fail(BF1_ERR_NO_DEVICE, "device compute capability %d.x is not sm_100", major);
-    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal));
-    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal));
-    // two CTAs per SM need the whole shared-memory carve-out
-    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                        cudaSharedmemCarveoutMaxShared));
-    BF1_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                        cudaSharedmemCarveoutMaxShared));
+    static bool configured[64] = {};
+    if (dev < 0 || dev >= 64) return fail(BF1_ERR_NO_DEVICE, "device ordinal %d out of range", dev);
+    if (!configured[dev]) {
+        // two CTAs per SM need the whole shared-memory carve-out
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal_dq));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal_dq));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal_kv));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal_kv));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+        configured[dev] = true;
+    }
     CUtensorMap tq, tk, tv, tg;
     // Q and dO: two heads and all column chunks per copy; with one head per KV head, one head and one chunk
     const int q_heads = group == 1 ? 1 : 2, q_chunks = group == 1 ? 1 : d / 64;
@@ -394,7 +743,9 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     if (int rc = make_map_4d(&tg, d_o, total_tokens, hq, d, q_heads, q_chunks)) return rc;
     if (int rc = make_map_4d(&tk, k, total_tokens, hkv, d, 1, d / 64)) return rc;
     if (int rc = make_map_4d(&tv, v, total_tokens, hkv, d, 1, d / 64)) return rc;
-    const size_t n_kv = (size_t)total_tokens * hkv * d;
+    const int cap = route->capacity_qblocks;
+    const BwdLayout lay(total_tokens, hq, hkv, d, cap, route->max_degree);
+    char* ws = (char*)workspace;
     BwdArgs a;
     a.cu_seqlens = cu_seqlens_dev;
     a.qb_seq = route->qb_seq;
@@ -403,7 +754,7 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.kv_idx = route->kv_idx;
     a.num_qblocks = route->num_qblocks;
     a.max_degree = route->max_degree;
-    a.capacity = route->capacity_qblocks;
+    a.capacity = cap;
     a.total_tokens = (int32_t)total_tokens;
     a.hq = hq;
     a.hkv = hkv;
@@ -414,16 +765,43 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.o = (const __nv_bfloat16*)o;
     a.d_o = (const __nv_bfloat16*)d_o;
     a.lse = lse;
+    a.delta = (float*)(ws + lay.delta);
     a.dq = (__nv_bfloat16*)dq;
-    a.dk32 = (float*)workspace;
-    a.dv32 = a.dk32 + n_kv;
+    a.dk = (__nv_bfloat16*)dk;
+    a.dv = (__nv_bfloat16*)dv;
+    a.partial = (float*)(ws + lay.partial);
+    int32_t* ip = (int32_t*)(ws + lay.ints);
+    a.inv.count = ip;            ip += lay.n_count;
+    a.inv.start = ip;            ip += lay.n_start;
+    a.inv.chunks = ip;           ip += lay.n_chunks;
+    a.inv.part0 = ip;            ip += lay.n_part0;
+    a.inv.wofs = ip;             ip += lay.n_wofs;
+    a.inv.readers = ip;          ip += lay.n_readers;
+    a.inv.unit_slot = ip;        ip += lay.n_units;
+    a.inv.unit_begin = ip;       ip += lay.n_units;
+    a.inv.unit_end = ip;         ip += lay.n_units;
+    a.inv.unit_part = ip;        ip += lay.n_units;
+    a.inv.scalars = ip;
+    a.inv.cap = cap;
+    a.inv.max_units = (int32_t)lay.n_units;
     cudaStream_t st = (cudaStream_t)stream;
-    BF1_CUDA_CHECK(cudaMemsetAsync(workspace, 0, 2 * n_kv * sizeof(float), st));
-    dim3 grid(route->capacity_qblocks, hkv, group == 4 ? 2 : 1);   // z: pairs of query heads
-    if (d == 128) attn_bwd_kernel<128><<<grid, kBwdThreads, BwdSmem<128>::kTotal, st>>>(tq, tk, tv, tg, a);
-    else attn_bwd_kernel<64><<<grid, kBwdThreads, BwdSmem<64>::kTotal, st>>>(tq, tk, tv, tg, a);
+    // the inverse route (readers of every KV block, cut into units) ...
+    inverse_route_kernel<false><<<cap, 256, 0, st>>>(a);
+    inverse_units_kernel<<<1, 1024, 0, st>>>(a);
+    inverse_route_kernel<true><<<cap, 256, 0, st>>>(a);
     BF1_CUDA_CHECK(cudaGetLastError());
-    bwd_round_kernel<<<296, 512, 0, st>>>(a.dk32, a.dv32, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, n_kv);
+    // ... dQ (and D_i) along the route, dK / dV along its inverse
+    dim3 grid_q(cap, hkv, group == 4 ? 2 : 1);   // z: pairs of query heads
+    dim3 grid_kv((unsigned)lay.n_units, hkv);
+    if (d == 128) {
+        bwd_dq_kernel<128><<<grid_q, kBwdThreads, BwdSmem<128>::kTotal_dq, st>>>(tq, tk, tv, tg, a);
+        bwd_dkv_kernel<128><<<grid_kv, kBwdThreads, BwdSmem<128>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
+        bwd_combine_kernel<128><<<dim3(cap, hkv), 256, 0, st>>>(a);
+    } else {
+        bwd_dq_kernel<64><<<grid_q, kBwdThreads, BwdSmem<64>::kTotal_dq, st>>>(tq, tk, tv, tg, a);
+        bwd_dkv_kernel<64><<<grid_kv, kBwdThreads, BwdSmem<64>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
+        bwd_combine_kernel<64><<<dim3(cap, hkv), 256, 0, st>>>(a);
+    }
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
 }

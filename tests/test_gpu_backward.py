@@ -1,7 +1,7 @@
-"""Gradients of the routed attention on the GPU vs the fp64 CPU oracle (Section 4.2: "forward and
-backward with finite Q/K/V gradients").  The kernel rounds P and dS to bf16 before its MMAs and
-its outputs to bf16, and adds dK / dV contributions with floating-point atomics, so the comparison
-is by relative RMS and by the largest error relative to the gradient's scale."""
+"""Gradients of the routed attention on the GPU vs the fp64 CPU oracle (Section 4.2's gradient gate).  The
+kernels round P and dS to bf16 before their MMAs and their outputs to bf16, so the comparison is by relative RMS
+and by the largest error relative to the gradient's scale.  Nothing is added with atomics: the three gradients
+must come out bit-identical on every run."""
 import numpy as np
 import pytest
 import torch
@@ -89,6 +89,42 @@ def test_gradients_in_every_geometry_the_forward_takes(hq, hkv, d):
         print(hq, hkv, d, lens, res)
         for name, (rms, mx) in res.items():
             assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
+
+
+@pytest.mark.parametrize("route", [dict(local_blocks=9, global_first=0, dyadic=0),      # sliding window: ten readers per block
+                                   dict(local_blocks=40, global_first=1, dyadic=1),     # 41+ readers per block: cut into runs
+                                   dict(local_blocks=0, global_first=0, dyadic=1)],     # dyadic predecessors only
+                         ids=["sliding", "wide", "dyadic-only"])
+def test_gradients_over_other_routes(route):
+    """dK / dV walk the INVERSE of whatever lists the route holds; these routes give it other shapes than BF1's."""
+    w = I.custom([4096, 700], hq=4, hkv=2, d=128, seed=6400, **route)
+    res = run_case(w, seed=5)
+    print(route, res)
+    for name, (rms, mx) in res.items():
+        assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
+
+
+def test_backward_is_bitwise_reproducible():
+    """No floating-point atomics: two runs give the same bits, whatever the workspace held before (block 0 of the
+    long sequence has 64 readers and goes through the partial-sum path)."""
+    dev = torch.device("cuda:0")
+    w = I.custom([4096, 1000, 65], hq=8, hkv=2, d=128, seed=6500)
+    q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+    d_o = torch.randn(q.shape, generator=torch.Generator().manual_seed(6)).to(torch.bfloat16).to(dev)
+    cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+    route = bf1.plan_route(cu, w.max_seqlen)
+    o, lse = bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route)
+    ws = bf1.bwd_workspace(route, w.total_tokens, w.hq, w.hkv, w.d, dev)
+    runs = []
+    for fill in (0x00, 0xFF, 0x7F):          # 0xFF bytes are NaNs as fp32, 0x7F.. huge ints as counters
+        ws.fill_(fill)
+        runs.append(bf1.attn_bwd(q, k, v, o, lse, d_o, cu, w.max_seqlen, route, workspace=ws))
+        torch.cuda.synchronize()
+        route.check_status()
+    for other in runs[1:]:
+        for x, y in zip(runs[0], other):
+            assert torch.equal(x, y)
+    assert all(torch.isfinite(t.float()).all() for t in runs[0])
 
 
 def test_backward_rejects_what_it_does_not_support():
