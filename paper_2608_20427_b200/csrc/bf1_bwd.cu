@@ -638,7 +638,8 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_co
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
-// KV blocks whose readers were cut into several runs: add the runs' partial sums in run order.
+// KV blocks whose readers were cut into several runs: add the runs' partial sums in run order.  Few blocks
+// need it (block 0 of a sequence, with the paper's route), so each is spread over gridDim.z CTAs by key rows.
 template <int D>
 __global__ void __launch_bounds__(256) bwd_combine_kernel(const BwdArgs a) {
     const int gp = blockIdx.x, kvh = blockIdx.y;
@@ -648,8 +649,11 @@ __global__ void __launch_bounds__(256) bwd_combine_kernel(const BwdArgs a) {
     const int seq = a.qb_seq[gp], p = a.qb_block[gp];
     const int seq0 = a.cu_seqlens[seq];
     const int kv_valid = min(kBlock64, a.cu_seqlens[seq + 1] - seq0 - p * kBlock64);
-    for (int i = threadIdx.x; i < kv_valid * D; i += 256) {
+    const int rows_per_cta = (kBlock64 + gridDim.z - 1) / gridDim.z;
+    const int i_lo = blockIdx.z * rows_per_cta * D, i_hi = min(kv_valid, (int)(blockIdx.z + 1) * rows_per_cta) * D;
+    for (int i = i_lo + threadIdx.x; i < i_hi; i += 256) {
         float sk = 0.f, sv = 0.f;
+#pragma unroll 4
         for (int r = 0; r < runs; ++r) {
             const float* pk = a.partial + (((size_t)(q0 + r) * a.hkv + kvh) * 2) * (kBlock64 * D);
             sk += pk[i];
@@ -796,11 +800,11 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     if (d == 128) {
         bwd_dq_kernel<128><<<grid_q, kBwdThreads, BwdSmem<128>::kTotal_dq, st>>>(tq, tk, tv, tg, a);
         bwd_dkv_kernel<128><<<grid_kv, kBwdThreads, BwdSmem<128>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
-        bwd_combine_kernel<128><<<dim3(cap, hkv), 256, 0, st>>>(a);
+        bwd_combine_kernel<128><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     } else {
         bwd_dq_kernel<64><<<grid_q, kBwdThreads, BwdSmem<64>::kTotal_dq, st>>>(tq, tk, tv, tg, a);
         bwd_dkv_kernel<64><<<grid_kv, kBwdThreads, BwdSmem<64>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
-        bwd_combine_kernel<64><<<dim3(cap, hkv), 256, 0, st>>>(a);
+        bwd_combine_kernel<64><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     }
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
