@@ -13,8 +13,8 @@
 //                    heads are the 128 rows of every MMA.  Per list entry p:
 //                        S  = Q  K_p^T   (128 x 64 x d)    A, B K-major from shared memory
 //                        dP = dO V_p^T   (128 x 64 x d)
-//                        dQ += dS K_p    (128 x d x 64)    A = dS (bf16, written to shared memory by the
-//                                                          threads), B = K_p MN-major; accumulates in TMEM
+//                        dQ += dS K_p    (128 x d x 64)    A = dS (bf16, written over S in tensor memory by
+//                                                          the threads), B = K_p MN-major; accumulates in TMEM
 //                    It also leaves D_i in the workspace for the second kernel.
 //   bwd_dkv_kernel   unit = (KV block p, KV head, a run of the query blocks that read p): the INVERSE
 //                    route, which three small kernels derive from the lists on every call (any lists: the
@@ -26,8 +26,8 @@
 //                    is cut into runs of `chunk` readers handled by different CTAs; their fp32 partial
 //                    sums are added in run order by bwd_combine_kernel.
 //
-// Both compute kernels are one CTA per unit, two CTAs per SM, every step of a tile in sequence; P is
-// rounded to bf16 before the MMAs, as in the forward.  With d = 64 the transposed products still run as
+// Both compute kernels are one CTA per unit, two CTAs per SM: four warps work on the tile rows, two issue copies
+// and one issues MMAs; P is rounded to bf16 before the MMAs, as in the forward.  With d = 64 the transposed products still run as
 // M = 128 MMAs: tensor-memory lanes 64..127 then hold nothing of value and are not read.
 #include <cuda.h>
 
@@ -36,7 +36,10 @@
 namespace bf1 {
 
 constexpr int kBlock64 = 64;     // b: tokens per block
-constexpr int kBwdThreads = 128;
+constexpr int kRowThreads = 128;               // threads that work on a tile's 128 rows
+constexpr int kPerRow = kRowThreads / 128;     // two per row: each takes 32 of a tile's 64 key columns
+constexpr int kRowWarps = kRowThreads / 32;
+constexpr int kBwdThreads = kRowThreads + 96;  // + two copy warps and one MMA warp
 constexpr int kMinChunk = 16;    // readers per dK/dV unit, at least
 
 // The inverse route and the units of bwd_dkv_kernel, all inside the caller's workspace.
@@ -92,14 +95,14 @@ struct BwdSmem {
     static constexpr int kDO = kQ + kQBytes;
     static constexpr int kK = kDO + kQBytes;
     static constexpr int kV = kK + kKVBytes;
-    // P and dS: [128 q rows][64 kv] bf16, 128-byte rows, swizzled (16 KB each).
-    //   dQ kernel:    only dS is needed; it has room of its own.
-    //   dK/dV kernel: at d = 128, P takes over V's buffer and dS takes over K's once S and dP have been
-    //                 computed (K and V are fetched again for the next reader; they come from L2); at d = 64 the
-    //                 K / V tiles are only 8 KB, so P and dS get room of their own.
-    static constexpr int kDS_dq = kV + kKVBytes;
-    static constexpr int kBar_dq = kDS_dq + 16384;
-    static constexpr int kTotal_dq = kBar_dq + 64;
+    // dQ kernel: dS goes to tensor memory, not to shared memory; the room it leaves is a second K buffer, so that
+    // the next K tile travels while the current one is in use (V is only needed for dP and is refetched early).
+    static constexpr int kK1_dq = kV + kKVBytes;
+    static constexpr int kBar_dq = kK1_dq + kKVBytes;
+    static constexpr int kTotal_dq = kBar_dq + 96;
+    // dK/dV kernel: P and dS [128 q rows][64 kv] bf16, 128-byte rows, swizzled (16 KB each).  At d = 128, P takes
+    // over V's buffer and dS takes over K's once S and dP have been computed (K and V are fetched again for the
+    // next reader; they come from L2); at d = 64 the K / V tiles are only 8 KB, so P and dS get room of their own.
     static constexpr int kP_kv = D == 128 ? kV : kV + kKVBytes;
     static constexpr int kDS_kv = D == 128 ? kK : kP_kv + 16384;
     static constexpr int kBar_kv = D == 128 ? kV + kKVBytes : kDS_kv + 16384;
@@ -116,55 +119,55 @@ __device__ __forceinline__ void issue_s_dp(uint32_t t_s, uint32_t t_dp, uint32_t
 #pragma unroll
     for (int kk = 0; kk < D / 16; ++kk) {
         const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
-        if (kk == 0) {
-            mma_ss_lohi<false>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
-            mma_ss_lohi<false>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
-        } else {
-            mma_ss_lohi<true>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
-            mma_ss_lohi<true>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
-        }
+        if (kk == 0) mma_ss_lohi<false>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
+        else mma_ss_lohi<true>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
+    }
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
+        if (kk == 0) mma_ss_lohi<false>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
+        else mma_ss_lohi<true>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
     }
 }
 
-// P and dS of this thread's row from S and dP in tensor memory, written as bf16 rows (128-byte rows, 16-byte
-// chunks XOR-swizzled with the row) where the next MMAs read them.  Masked entries get s = -inf (self block,
-// warp-uniform branch) and rows outside the sequence an infinite LSE: both give P = 0 exactly, and with it dS = 0.
-template <bool kWriteP>
-__device__ __forceinline__ void p_and_ds(uint32_t t_s, uint32_t t_dp, uint32_t prow, uint32_t dsrow, int tid, int tl, bool diag,
-                                         float lse_row2, float drow, float scale, float scale_log2) {
+// P and dS of this thread's 32 columns (half = 0 / 1: columns 0..31 / 32..63) of its row, from S and dP in tensor
+// memory.  Masked entries get s = -inf (self block, warp-uniform branch) and rows outside the sequence an infinite
+// LSE: both give P = 0 exactly, and with it dS = 0.  Results as packed bf16 pairs.
+__device__ __forceinline__ void p_and_ds(uint32_t t_s, uint32_t t_dp, int half, int tl, bool diag, float lse_row2, float drow,
+                                         float scale, float scale_log2, uint32_t (&pw)[16], uint32_t (&dw)[16]) {
     const uint64_t c2p = pack2(scale_log2, scale_log2), nlp = pack2(-lse_row2, -lse_row2);
     const uint64_t scp = pack2(scale, scale), ndp = pack2(-drow * scale, -drow * scale);
+    uint32_t sr[32], dr[32];
+    tmem_ld32(t_s + half * 32, sr);
+    tmem_ld32(t_dp + half * 32, dr);
+    tmem_wait_ld();
+    if (diag) {
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        uint32_t sr[32], dr[32];
-        tmem_ld32(t_s + half * 32, sr);
-        tmem_ld32(t_dp + half * 32, dr);
-        tmem_wait_ld();
-        if (diag) {
+        for (int c = 0; c < 32; ++c)
+            if (half * 32 + c > tl) sr[c] = 0xff800000u;   // -inf: causal triangle
+    }
 #pragma unroll
-            for (int c = 0; c < 32; ++c)
-                if (half * 32 + c > tl) sr[c] = 0xff800000u;   // -inf: causal triangle
-        }
-        uint32_t pw[16], dw[16];
+    for (int c = 0; c < 16; ++c) {
+        const uint64_t x = fma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), c2p, nlp);
+        float x0, x1;
+        unpack2(x, x0, x1);
+        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+        // dS = P * (dP - D) * scale
+        const uint64_t t = fma2(pack2(__uint_as_float(dr[2 * c]), __uint_as_float(dr[2 * c + 1])), scp, ndp);
+        float d0, d1;
+        unpack2(mul2(pack2(p0, p1), t), d0, d1);
+        pw[c] = pack_bf16x2(p0, p1);
+        dw[c] = pack_bf16x2(d0, d1);
+    }
+}
+
+// The same pairs as a bf16 row piece in shared memory: 128-byte rows, 16-byte chunks XOR-swizzled with the row
+// (the layout the MMAs read as an MN-major operand).
+__device__ __forceinline__ void store_row_piece(uint32_t row_addr, int row, int half, const uint32_t (&w)[16]) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            const uint64_t x = fma2(pack2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), c2p, nlp);
-            float x0, x1;
-            unpack2(x, x0, x1);
-            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-            // dS = P * (dP - D) * scale
-            const uint64_t t = fma2(pack2(__uint_as_float(dr[2 * c]), __uint_as_float(dr[2 * c + 1])), scp, ndp);
-            float d0, d1;
-            unpack2(mul2(pack2(p0, p1), t), d0, d1);
-            pw[c] = pack_bf16x2(p0, p1);
-            dw[c] = pack_bf16x2(d0, d1);
-        }
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk half * 4 + c4 of the 128-byte row
-            const int ch = (half * 4 + c4) ^ (tid & 7);
-            if (kWriteP) st_shared_v4(prow + (ch << 4), pw[4 * c4], pw[4 * c4 + 1], pw[4 * c4 + 2], pw[4 * c4 + 3]);
-            st_shared_v4(dsrow + (ch << 4), dw[4 * c4], dw[4 * c4 + 1], dw[4 * c4 + 2], dw[4 * c4 + 3]);
-        }
+    for (int c4 = 0; c4 < 4; ++c4) {                          // 16-byte chunk half * 4 + c4 of the 128-byte row
+        const int ch = (half * 4 + c4) ^ (row & 7);
+        st_shared_v4(row_addr + (ch << 4), w[4 * c4], w[4 * c4 + 1], w[4 * c4 + 2], w[4 * c4 + 3]);
     }
 }
 
@@ -179,36 +182,42 @@ __device__ __forceinline__ void clear_idle_rows(uint32_t sQ, uint32_t sDO, int t
     fence_proxy_async();
 }
 
-// Q and dO tiles of one query block and pair of heads (thread 0 only; expect_tx is the caller's).
+// One Q-shaped tile (Q, dO or O) of a query block and pair of heads (one thread; expect_tx is the caller's).
 template <int D>
-__device__ __forceinline__ void load_q_do(uint32_t sQ, uint32_t sDO, const CUtensorMap* tm_q, const CUtensorMap* tm_do, int tok0,
-                                          int head, int group, uint32_t bar) {
+__device__ __forceinline__ void load_q_tile(uint32_t dst, const CUtensorMap* tm, int tok0, int head, int group, uint32_t bar) {
     if (group > 1) {
-        tma_load_4d(sQ, tm_q, 0, tok0, head, 0, bar);
-        tma_load_4d(sDO, tm_do, 0, tok0, head, 0, bar);
+        tma_load_4d(dst, tm, 0, tok0, head, 0, bar);
     } else {
 #pragma unroll
-        for (int ch = 0; ch < D / 64; ++ch) {
-            tma_load_4d(sQ + ch * 16384, tm_q, 0, tok0, head, ch, bar);
-            tma_load_4d(sDO + ch * 16384, tm_do, 0, tok0, head, ch, bar);
-        }
+        for (int ch = 0; ch < D / 64; ++ch) tma_load_4d(dst + ch * 16384, tm, 0, tok0, head, ch, bar);
     }
 }
 
+__device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t (&w)[4]) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+}
+
 // ---- dQ --------------------------------------------------------------------------------------------------------
+
+// Warp roles of the two compute kernels: the row warps do the arithmetic on S and dP (one or two threads per tile
+// row), two warps issue copies (one thread keeps a TMA queue only about half full) and one issues MMAs.  Nobody
+// but the row warps ever waits for arithmetic, so copies and MMAs of the next list entry are under way while the
+// current one is being worked on.
+constexpr int kWarpLoadA = kRowWarps, kWarpLoadB = kRowWarps + 1, kWarpMma = kRowWarps + 2;
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                              const __grid_constant__ CUtensorMap tm_k,
                                                              const __grid_constant__ CUtensorMap tm_v,
                                                              const __grid_constant__ CUtensorMap tm_do,
+                                                             const __grid_constant__ CUtensorMap tm_o,
                                                              const BwdArgs a) {
     using L = BwdSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     // no static shared memory: it would cost a whole extra kilobyte and with it the second CTA per SM
-    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_dq + 40);
-    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_dq + 44);
-    const int tid = threadIdx.x, warp = tid >> 5;
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_dq + 88);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_dq + 92);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = blockIdx.x, kvh = blockIdx.y, pair = blockIdx.z;   // pair: which two query heads of the group
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
     if (slot >= min(*a.num_qblocks, a.capacity)) return;
@@ -221,16 +230,26 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_kernel(const __grid_con
     const int tok0 = seq0 + j * kBlock64;
 
     const uint32_t base = smem_u32(smem);
-    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV, sDS = base + L::kDS_dq;
-    const uint32_t bar_q = base + L::kBar_dq, bar_k = bar_q + 8, bar_v = bar_q + 16, bar_a = bar_q + 24, bar_b = bar_q + 32;
+    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sV = base + L::kV;
+    const uint32_t sO = sV;   // the O tile lies over V and the second K buffer until D_i has been computed
+    const uint32_t sKbuf[2] = {base + L::kK, base + L::kK1_dq};
+    // bar_q: Q, dO, O landed; bar_k[2], bar_v: a K / V tile landed; bar_sdp: S and dP computed; bar_ds: dS written
+    // (one arrival per row warp); bar_dq[2]: the dQ MMAs of an entry done (alternating, like the K buffers they
+    // free); bar_o: the O tile has been read (one arrival per row warp)
+    const uint32_t bar_q = base + L::kBar_dq, bar_k = bar_q + 8 /* [2] */, bar_v = bar_q + 24, bar_sdp = bar_q + 32,
+                   bar_ds = bar_q + 40, bar_dq = bar_q + 48 /* [2] */, bar_o = bar_q + 64;
     if (tid == 0) {
         s_abort = (base & 1023u) ? 1 : 0;
         if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
-        mbar_init(bar_q, 1);
+        mbar_init(bar_q, 2);
         mbar_init(bar_k, 1);
+        mbar_init(bar_k + 8, 1);
         mbar_init(bar_v, 1);
-        mbar_init(bar_a, 1);
-        mbar_init(bar_b, 1);
+        mbar_init(bar_sdp, 1);
+        mbar_init(bar_ds, kRowWarps);
+        mbar_init(bar_dq, 1);
+        mbar_init(bar_dq + 8, 1);
+        mbar_init(bar_o, kRowWarps);
         fence_mbar_init();
     }
     __syncwarp();
@@ -244,111 +263,171 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_kernel(const __grid_con
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* abort_flag = &s_abort;
+    if (s_abort) {   // (uniform over the CTA)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, 256);
+        return;
+    }
+    // S and dP: 64 fp32 columns each; dS (bf16 pairs) takes over columns 0..15 and 32..47 of S; dQ: d columns
     constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128;
-    const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    constexpr uint32_t kQTx = L::kQBytes;
+    const int head0 = kvh * a.group + pair * 2;
+    const uint32_t q_tx = a.group > 1 ? kQTx : kQTx / 2;   // one head per KV head: half a tile per copy set
 
-    // rows of this thread: head hl, token tl of the query block
-    const int hl = tid >> 6, tl = tid & 63;
-    const int h = kvh * a.group + pair * 2 + hl;
-    const int tok = tok0 + tl;
-    const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;   // G = 1: rows 64..127 belong to no head
-
-    // K and V have a barrier each: V is free as soon as dP has been computed, K only after dQ += dS K
-    auto load_k = [&](int p) {   // thread 0 only
-        mbar_expect_tx(bar_k, L::kKVBytes);
-        tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_k);
-    };
-    auto load_v = [&](int p) {
-        mbar_expect_tx(bar_v, L::kKVBytes);
-        tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_v);
-    };
-    if (tid == 0 && !s_abort) {
-        mbar_expect_tx(bar_q, a.group > 1 ? 2 * L::kQBytes : L::kQBytes);
-        load_q_do<D>(sQ, sDO, &tm_q, &tm_do, tok0, kvh * a.group + pair * 2, a.group, bar_q);
+    if (warp == kWarpLoadA) {
+        // ---- copies, first half: dO, Q, then the K tiles (tile `it` in buffer it & 1, fetched two entries ahead) ----
         const int p0 = list_entry(list, 0, cnt, j);
-        load_k(p0);
-        load_v(p0);
-    }
-    // D_i = <dO_i, O_i> and the row's LSE in the log2 domain
-    float Drow = 0.f, lse2 = INFINITY;
-    if (row_ok) {
-        const uint4* op = reinterpret_cast<const uint4*>(a.o + ((size_t)tok * a.hq + h) * D);
-        const uint4* gp = reinterpret_cast<const uint4*>(a.d_o + ((size_t)tok * a.hq + h) * D);
-#pragma unroll 4
-        for (int c = 0; c < D / 8; ++c) {
-            const uint4 ov = op[c], gv = gp[c];
-            const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                Drow = fmaf(__uint_as_float(ow[e] << 16), __uint_as_float(gw[e] << 16), Drow);
-                Drow = fmaf(__uint_as_float(ow[e] & 0xffff0000u), __uint_as_float(gw[e] & 0xffff0000u), Drow);
-            }
+        if (elect_one()) {
+            mbar_expect_tx(bar_q, 2 * q_tx);
+            load_q_tile<D>(sDO, &tm_do, tok0, head0, a.group, bar_q);
+            load_q_tile<D>(sQ, &tm_q, tok0, head0, a.group, bar_q);
+            mbar_expect_tx(bar_k, L::kKVBytes);
+            tma_load_4d(sKbuf[0], &tm_k, 0, seq0 + p0 * kBlock64, kvh, 0, bar_k);
         }
-        lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
-        a.delta[(size_t)h * a.total_tokens + tok] = Drow;   // for the dK/dV kernel
-    }
-    mbar_wait(bar_q, 0, abort_flag, a.status);
-
-    constexpr uint32_t kHi = desc_hi_sw128(1024);
-    constexpr uint32_t kIdQ = idesc_bf16_f32_ab(D, false, true);       // dQ: 128 x d, B (K tile) MN-major
-    for (int it = 0; it < cnt; ++it) {
-        const int p_next = (it + 1 < cnt) ? list_entry(list, it + 1, cnt, j) : 0;
-        const bool diag = (it == cnt - 1);
-        if (tid == 0) {
-            mbar_wait(bar_k, it & 1, abort_flag, a.status);
+        __syncwarp();
+        if (cnt > 1) {
+            const int p1 = list_entry(list, 1, cnt, j);
+            mbar_wait(bar_o, 0, abort_flag, a.status);
+            if (elect_one()) {
+                mbar_expect_tx(bar_k + 8, L::kKVBytes);
+                tma_load_4d(sKbuf[1], &tm_k, 0, seq0 + p1 * kBlock64, kvh, 0, bar_k + 8);
+            }
+            __syncwarp();
+        }
+        for (int it = 0; it + 2 < cnt; ++it) {
+            const int p = list_entry(list, it + 2, cnt, j);
+            mbar_wait(bar_dq + 8 * (it & 1), (it >> 1) & 1, abort_flag, a.status);   // dQ(it) done: its K buffer is free
+            if (elect_one()) {
+                mbar_expect_tx(bar_k + 8 * (it & 1), L::kKVBytes);
+                tma_load_4d(sKbuf[it & 1], &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_k + 8 * (it & 1));
+            }
+            __syncwarp();
+        }
+    } else if (warp == kWarpLoadB) {
+        // ---- copies, second half: O, then the V tiles (one buffer, refetched as soon as dP has been computed) ----
+        if (elect_one()) {
+            mbar_expect_tx(bar_q, q_tx);
+            load_q_tile<D>(sO, &tm_o, tok0, head0, a.group, bar_q);
+        }
+        __syncwarp();
+        for (int it = 0; it < cnt; ++it) {
+            const int p = list_entry(list, it, cnt, j);
+            if (it == 0) mbar_wait(bar_o, 0, abort_flag, a.status);
+            else mbar_wait(bar_sdp, (it - 1) & 1, abort_flag, a.status);
+            if (elect_one()) {
+                mbar_expect_tx(bar_v, L::kKVBytes);
+                tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_v);
+            }
+            __syncwarp();
+        }
+    } else if (warp == kWarpMma) {
+        // ---- MMAs: S, dP of entry it + 1 are issued right behind dQ of entry it (the pipe runs them in order, so the
+        // new S only overwrites dS once the dQ MMAs have read it) ----
+        constexpr uint32_t kHi = desc_hi_sw128(1024);
+        constexpr uint32_t kIdQ = idesc_bf16_f32(D, true);             // dQ: 128 x d, A from tensor memory, B (K tile) MN-major
+        mbar_wait(bar_q, 0, abort_flag, a.status);
+        for (int it = 0; it < cnt; ++it) {
+            const int kb = it & 1;
+            mbar_wait(bar_k + 8 * kb, (it >> 1) & 1, abort_flag, a.status);
             mbar_wait(bar_v, it & 1, abort_flag, a.status);
             tc_fence_after();
-            issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sK, sV);
-            mma_commit(bar_a);
-        }
-        __syncwarp();
-        mbar_wait(bar_a, it & 1, abort_flag, a.status);
-        tc_fence_after();
-        if (tid == 0 && it + 1 < cnt) load_v(p_next);   // V is free: its next tile travels during the arithmetic below
-        p_and_ds<false>(t_lane + kColS, t_lane + kColDP, 0u, sDS + tid * 128, tid, tl, diag, lse2, Drow, a.scale, a.scale_log2);
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-
-        if (tid == 0) {
-            tc_fence_after();
-            // dQ += dS K: A = dS [128 q][64 kv] K-major (4 k-steps of 16 kv = 32 bytes), B = K tile MN-major
-            // (16 kv rows = 2048 bytes per step, next 64 d columns 8 KB away)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {   // 64 kv rows in steps of 16
-                const uint32_t alo = desc_lo_sw128(sDS, 16) + ((kk * 32) >> 4);
-                const uint32_t blo = desc_lo_sw128(sK, 8192) + ((kk * 2048) >> 4);
-                if (it == 0 && kk == 0) mma_ss_lohi<false>(tmem + kColDQ, alo, blo, kHi, kIdQ);
-                else mma_ss_lohi<true>(tmem + kColDQ, alo, blo, kHi, kIdQ);
+            if (elect_one()) {
+                issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sKbuf[kb], sV);
+                mma_commit(bar_sdp);
             }
-            mma_commit(bar_b);
-        }
-        __syncwarp();
-        mbar_wait(bar_b, it & 1, abort_flag, a.status);   // K, the dS buffer and the S / dP columns are free again
-        tc_fence_after();
-        if (tid == 0 && it + 1 < cnt) load_k(p_next);
-    }
-
-    // ---- dQ rows -----------------------------------------------------------------------------------
-    __nv_bfloat16* dqrow = a.dq + ((size_t)tok * a.hq + h) * D;
+            __syncwarp();
+            mbar_wait(bar_ds, it & 1, abort_flag, a.status);
+            tc_fence_after();
+            if (elect_one()) {
+                // dQ += dS K: A = dS [128 q][64 kv] from tensor memory (16 kv = 8 columns per step; keys 0..31 sit in
+                // columns 0..15, keys 32..63 in columns 32..47), B = K tile MN-major (16 kv rows = 2048 bytes per step,
+                // next 64 d columns 8 KB away)
 #pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(t_lane + kColDQ + c * 32, r);
-        tmem_wait_ld();
+                for (int kk = 0; kk < 4; ++kk) {   // 64 kv rows in steps of 16
+                    const uint32_t blo = desc_lo_sw128(sKbuf[kb], 8192) + ((kk * 2048) >> 4);
+                    const uint32_t a_ds = tmem + kColS + (kk >> 1) * 32 + (kk & 1) * 8;
+                    if (it == 0 && kk == 0) mma_ts_lohi<false>(tmem + kColDQ, a_ds, blo, kHi, kIdQ);
+                    else mma_ts_lohi<true>(tmem + kColDQ, a_ds, blo, kHi, kIdQ);
+                }
+                mma_commit(bar_dq + 8 * kb);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ---- row warps: tile row (head hl, token tl of the query block) and which half of a tile's 64 key columns ----
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const int row = tid & 127, half = tid >> 7;
+        const int hl = row >> 6, tl = row & 63;
+        const int h = head0 + hl;
+        const int tok = tok0 + tl;
+        const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;   // G = 1: rows 64..127 belong to no head
+        // D_i = <dO_i, O_i> from the two tiles in shared memory (both threads of a row compute it), and the row's
+        // LSE in the log2 domain
+        float lse2 = INFINITY;
+        if (row_ok) lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
+        mbar_wait(bar_q, 0, abort_flag, a.status);
+        float Drow = 0.f;
         if (row_ok) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-                uint4 w;
-                w.x = pack_bf16x2(__uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
-                w.y = pack_bf16x2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                w.z = pack_bf16x2(__uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
-                w.w = pack_bf16x2(__uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
-                *reinterpret_cast<uint4*>(dqrow + c * 32 + e) = w;
+            for (int c = 0; c < D / 8; ++c) {   // 16-byte pieces of the row: chunk c / 8 of 64 columns, piece c % 8
+                const uint32_t off = (c >> 3) * 16384 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                uint32_t ow[4], gw[4];
+                ld_shared_v4(sO + off, ow);
+                ld_shared_v4(sDO + off, gw);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    Drow = fmaf(__uint_as_float(ow[e] << 16), __uint_as_float(gw[e] << 16), Drow);
+                    Drow = fmaf(__uint_as_float(ow[e] & 0xffff0000u), __uint_as_float(gw[e] & 0xffff0000u), Drow);
+                }
+            }
+            if (half == 0) a.delta[(size_t)h * a.total_tokens + tok] = Drow;   // for the dK/dV kernel
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_o);
+
+        for (int it = 0; it < cnt; ++it) {
+            const bool diag = (it == cnt - 1);
+            mbar_wait(bar_sdp, it & 1, abort_flag, a.status);
+            tc_fence_after();
+            for (int hh = half * (2 / kPerRow); hh < (half + 1) * (2 / kPerRow); ++hh) {
+                uint32_t pw[16], dw[16];
+                p_and_ds(t_lane + kColS, t_lane + kColDP, hh, tl, diag, lse2, Drow, a.scale, a.scale_log2, pw, dw);
+                // dS as the A operand of the next MMA: bf16 pairs, written over the first 16 of the 32 S columns this
+                // thread has just read (its own columns only: the row's other thread may still be reading its half)
+                __syncwarp();
+                tmem_st16(t_lane + kColS + hh * 32, dw);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ds);
+        }
+        // the last dQ MMA
+        mbar_wait(bar_dq + 8 * ((cnt - 1) & 1), ((cnt - 1) >> 1) & 1, abort_flag, a.status);
+        tc_fence_after();
+
+        // ---- dQ rows: each of a row's threads stores its share of the columns ----
+        constexpr int kColsPerThread = D / kPerRow;
+        __nv_bfloat16* dqrow = a.dq + ((size_t)tok * a.hq + h) * D + half * kColsPerThread;
+#pragma unroll
+        for (int c = 0; c < kColsPerThread / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(t_lane + kColDQ + half * kColsPerThread + c * 32, r);
+            tmem_wait_ld();
+            if (row_ok) {
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
+                    w.y = pack_bf16x2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                    w.z = pack_bf16x2(__uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
+                    w.w = pack_bf16x2(__uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
+                    *reinterpret_cast<uint4*>(dqrow + c * 32 + e) = w;
+                }
             }
         }
+        tc_fence_before();
     }
-    tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
@@ -497,9 +576,9 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_co
                                                               const BwdArgs a) {
     using L = BwdSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_kv + 32);
-    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_kv + 36);
-    const int tid = threadIdx.x, warp = tid >> 5;
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_kv + 48);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_kv + 52);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int unit = blockIdx.x, kvh = blockIdx.y;
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
     if (unit >= a.inv.scalars[0]) return;
@@ -514,13 +593,17 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_co
     const uint32_t base = smem_u32(smem);
     const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV;
     const uint32_t sP = base + L::kP_kv, sDS = base + L::kDS_kv;
-    const uint32_t bar_ld = base + L::kBar_kv, bar_a = bar_ld + 8, bar_b = bar_ld + 16;
+    // bar_ld: the four tiles of a step landed (both copy warps announce their bytes); bar_sdp: S and dP computed;
+    // bar_pds: P and dS written (one arrival per row warp); bar_acc: the step's dV^T / dK^T MMAs done, every buffer
+    // is free again
+    const uint32_t bar_ld = base + L::kBar_kv, bar_sdp = bar_ld + 8, bar_pds = bar_ld + 16, bar_acc = bar_ld + 24;
     if (tid == 0) {
         s_abort = (base & 1023u) ? 1 : 0;
         if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
-        mbar_init(bar_ld, 1);
-        mbar_init(bar_a, 1);
-        mbar_init(bar_b, 1);
+        mbar_init(bar_ld, 2);
+        mbar_init(bar_sdp, 1);
+        mbar_init(bar_pds, kRowWarps);
+        mbar_init(bar_acc, 1);
         fence_mbar_init();
     }
     __syncwarp();
@@ -534,106 +617,139 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_co
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* abort_flag = &s_abort;
+    const int steps = (r_end - r_begin) * pairs;
+    if (s_abort || steps <= 0) {   // (uniform over the CTA)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, 256);
+        return;
+    }
     // S and dP are recomputed for every reader; dV^T and dK^T stay where they are until the last one
     constexpr uint32_t kColS = 0, kColDP = 64, kColDVt = 128, kColDKt = 192;
-    const uint32_t t_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-    const int hl = tid >> 6, tl = tid & 63;
-    constexpr uint32_t kHi = desc_hi_sw128(1024);
-    constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);       // dV^T, dK^T: A and B MN-major
+    const uint32_t q_tx = a.group > 1 ? L::kQBytes : L::kQBytes / 2;
 
-    const int steps = (r_end - r_begin) * pairs;
-    // thread 0 only: Q, dO of query block jq (a block of this block's own sequence) and pair; K, V of this block again
-    auto issue_loads = [&](int jq, int pair) {
-        mbar_expect_tx(bar_ld, (a.group > 1 ? 2 * L::kQBytes : L::kQBytes) + 2 * L::kKVBytes);
-        load_q_do<D>(sQ, sDO, &tm_q, &tm_do, seq0 + jq * kBlock64, kvh * a.group + pair * 2, a.group, bar_ld);
-        tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
-        tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
-    };
-    // the reader of a step and its block index are fetched one step ahead: two dependent global loads that
-    // would otherwise sit in front of every copy
-    int g_next = steps > 0 ? a.inv.readers[r_begin] : gp;
-    int jq_next = a.qb_block[g_next];
-    if (tid == 0 && !s_abort && steps > 0) issue_loads(jq_next, 0);
-    for (int step = 0; step < steps; ++step) {
-        const int g = g_next, jq = jq_next, pair = step % pairs;
-        if (step + 1 < steps) {
-            g_next = a.inv.readers[r_begin + (step + 1) / pairs];
-            jq_next = a.qb_block[g_next];
-        }
-        const int rows_valid = min(kBlock64, seqlen - jq * kBlock64);
-        const int h = kvh * a.group + pair * 2 + hl;
-        const int tok = seq0 + jq * kBlock64 + tl;
-        const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;
-        // the row's LSE (log2 domain) and D_i, fetched while the tiles travel
-        float lse2 = INFINITY, drow = 0.f;
-        if (row_ok) {
-            lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
-            drow = a.delta[(size_t)h * a.total_tokens + tok];
-        }
-        if (tid == 0) {
-            mbar_wait(bar_ld, step & 1, abort_flag, a.status);
-            tc_fence_after();
-            issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sK, sV);
-            mma_commit(bar_a);
-        }
-        __syncwarp();
-        mbar_wait(bar_a, step & 1, abort_flag, a.status);
-        tc_fence_after();
-        p_and_ds<true>(t_lane + kColS, t_lane + kColDP, sP + tid * 128, sDS + tid * 128, tid, tl, g == gp, lse2, drow, a.scale,
-                       a.scale_log2);
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            // dV^T += dO^T P and dK^T += Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
-            // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t ko = (kk * 2048) >> 4;
-                if (kk == 0 && step == 0) {
-                    mma_ss_lohi<false>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                    mma_ss_lohi<false>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+    if (warp == kWarpLoadA || warp == kWarpLoadB) {
+        // ---- copies: Q and K (first warp), dO and V (second warp) of every step.  P takes over V's buffer and dS
+        // K's at d = 128, so K and V come again for every reader (from L2). ----
+        const bool first = warp == kWarpLoadA;
+        int jq = a.qb_block[a.inv.readers[r_begin]];
+        for (int step = 0; step < steps; ++step) {
+            int jq_next = 0;
+            if (step + 1 < steps) jq_next = a.qb_block[a.inv.readers[r_begin + (step + 1) / pairs]];
+            if (step > 0) mbar_wait(bar_acc, (step - 1) & 1, abort_flag, a.status);
+            if (elect_one()) {
+                mbar_expect_tx(bar_ld, q_tx + L::kKVBytes);
+                const int head0 = kvh * a.group + (step % pairs) * 2;
+                if (first) {
+                    tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
+                    load_q_tile<D>(sQ, &tm_q, seq0 + jq * kBlock64, head0, a.group, bar_ld);
                 } else {
-                    mma_ss_lohi<true>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                    mma_ss_lohi<true>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                    tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
+                    load_q_tile<D>(sDO, &tm_do, seq0 + jq * kBlock64, head0, a.group, bar_ld);
                 }
             }
-            mma_commit(bar_b);
+            __syncwarp();
+            jq = jq_next;
         }
-        __syncwarp();
-        mbar_wait(bar_b, step & 1, abort_flag, a.status);   // every buffer is free again
+    } else if (warp == kWarpMma) {
+        constexpr uint32_t kHi = desc_hi_sw128(1024);
+        constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);   // dV^T, dK^T: A and B MN-major
+        for (int step = 0; step < steps; ++step) {
+            mbar_wait(bar_ld, step & 1, abort_flag, a.status);
+            tc_fence_after();
+            if (elect_one()) {
+                issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sK, sV);
+                mma_commit(bar_sdp);
+            }
+            __syncwarp();
+            mbar_wait(bar_pds, step & 1, abort_flag, a.status);
+            tc_fence_after();
+            if (elect_one()) {
+                // dV^T += dO^T P and dK^T += Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
+                // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t ko = (kk * 2048) >> 4;
+                    if (kk == 0 && step == 0) mma_ss_lohi<false>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                    else mma_ss_lohi<true>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t ko = (kk * 2048) >> 4;
+                    if (kk == 0 && step == 0) mma_ss_lohi<false>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                    else mma_ss_lohi<true>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                }
+                mma_commit(bar_acc);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ---- row warps: tile row (head hl, token tl of the reader) and which half of the 64 key columns ----
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const int row = tid & 127, half = tid >> 7;
+        const int hl = row >> 6, tl = row & 63;
+        // the reader of a step, its block index, the row's LSE (log2 domain) and D_i are fetched one step ahead:
+        // dependent global loads that would otherwise sit between the MMAs and the arithmetic
+        auto fetch = [&](int step, int& g, float& lse2, float& drow) {
+            g = a.inv.readers[r_begin + step / pairs];
+            const int jq = a.qb_block[g], pr = step % pairs;
+            const int rows_valid = min(kBlock64, seqlen - jq * kBlock64);
+            lse2 = INFINITY;
+            drow = 0.f;
+            if (tl < rows_valid && pr * 2 + hl < a.group) {
+                const size_t at = (size_t)(kvh * a.group + pr * 2 + hl) * a.total_tokens + seq0 + jq * kBlock64 + tl;
+                lse2 = a.lse[at] * 1.4426950408889634f;
+                drow = a.delta[at];
+            }
+        };
+        int g, g_next = 0;
+        float lse2, drow, lse2_next = INFINITY, drow_next = 0.f;
+        fetch(0, g, lse2, drow);
+        for (int step = 0; step < steps; ++step) {
+            if (step + 1 < steps) fetch(step + 1, g_next, lse2_next, drow_next);
+            mbar_wait(bar_sdp, step & 1, abort_flag, a.status);
+            tc_fence_after();
+            for (int hh = half * (2 / kPerRow); hh < (half + 1) * (2 / kPerRow); ++hh) {
+                uint32_t pw[16], dw[16];
+                p_and_ds(t_lane + kColS, t_lane + kColDP, hh, tl, g == gp, lse2, drow, a.scale, a.scale_log2, pw, dw);
+                store_row_piece(sP + row * 128, row, hh, pw);
+                store_row_piece(sDS + row * 128, row, hh, dw);
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_pds);
+            g = g_next, lse2 = lse2_next, drow = drow_next;
+        }
+        mbar_wait(bar_acc, (steps - 1) & 1, abort_flag, a.status);
         tc_fence_after();
-        if (tid == 0 && step + 1 < steps) issue_loads(jq_next, (step + 1) % pairs);
-    }
 
-    // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns -----------------------
-    if (tid < D && steps > 0) {   // d = 64: lanes 64..127 hold nothing (warp-uniform)
-        const size_t rstride = (size_t)a.hkv * D;
-        const size_t row0 = ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + tid;
-        float* pk = part >= 0 ? a.partial + (((size_t)part * a.hkv + kvh) * 2) * (kBlock64 * D) + tid : nullptr;
+        // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns ----
+        if (row < D) {   // d = 64: lanes 64..127 hold nothing (warp-uniform)
+            const size_t rstride = (size_t)a.hkv * D;
+            const size_t row0 = ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + row;
+            float* pk = part >= 0 ? a.partial + (((size_t)part * a.hkv + kvh) * 2) * (kBlock64 * D) + row : nullptr;
+            for (int hh = half * (2 / kPerRow); hh < (half + 1) * (2 / kPerRow); ++hh) {
+                uint32_t vr[32], kr[32];
+                tmem_ld32(t_lane + kColDVt + hh * 32, vr);
+                tmem_ld32(t_lane + kColDKt + hh * 32, kr);
+                tmem_wait_ld();
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t vr[32], kr[32];
-            tmem_ld32(t_lane + kColDVt + half * 32, vr);
-            tmem_ld32(t_lane + kColDKt + half * 32, kr);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const int kvr = half * 32 + c;
-                if (kvr < kv_valid) {
-                    if (part < 0) {
-                        a.dv[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(vr[c]));
-                        a.dk[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(kr[c]));
-                    } else {
-                        pk[kvr * D] = __uint_as_float(kr[c]);
-                        pk[kBlock64 * D + kvr * D] = __uint_as_float(vr[c]);
+                for (int c = 0; c < 32; ++c) {
+                    const int kvr = hh * 32 + c;
+                    if (kvr < kv_valid) {
+                        if (part < 0) {
+                            a.dv[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(vr[c]));
+                            a.dk[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(kr[c]));
+                        } else {
+                            pk[kvr * D] = __uint_as_float(kr[c]);
+                            pk[kBlock64 * D + kvr * D] = __uint_as_float(vr[c]);
+                        }
                     }
                 }
             }
         }
+        tc_fence_before();
     }
-    tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
@@ -740,11 +856,12 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
         configured[dev] = true;
     }
-    CUtensorMap tq, tk, tv, tg;
+    CUtensorMap tq, tk, tv, tg, to;
     // Q and dO: two heads and all column chunks per copy; with one head per KV head, one head and one chunk
     const int q_heads = group == 1 ? 1 : 2, q_chunks = group == 1 ? 1 : d / 64;
     if (int rc = make_map_4d(&tq, q, total_tokens, hq, d, q_heads, q_chunks)) return rc;
     if (int rc = make_map_4d(&tg, d_o, total_tokens, hq, d, q_heads, q_chunks)) return rc;
+    if (int rc = make_map_4d(&to, o, total_tokens, hq, d, q_heads, q_chunks)) return rc;
     if (int rc = make_map_4d(&tk, k, total_tokens, hkv, d, 1, d / 64)) return rc;
     if (int rc = make_map_4d(&tv, v, total_tokens, hkv, d, 1, d / 64)) return rc;
     const int cap = route->capacity_qblocks;
@@ -798,11 +915,11 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     dim3 grid_q(cap, hkv, group == 4 ? 2 : 1);   // z: pairs of query heads
     dim3 grid_kv((unsigned)lay.n_units, hkv);
     if (d == 128) {
-        bwd_dq_kernel<128><<<grid_q, kBwdThreads, BwdSmem<128>::kTotal_dq, st>>>(tq, tk, tv, tg, a);
+        bwd_dq_kernel<128><<<grid_q, kBwdThreads, BwdSmem<128>::kTotal_dq, st>>>(tq, tk, tv, tg, to, a);
         bwd_dkv_kernel<128><<<grid_kv, kBwdThreads, BwdSmem<128>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
         bwd_combine_kernel<128><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     } else {
-        bwd_dq_kernel<64><<<grid_q, kBwdThreads, BwdSmem<64>::kTotal_dq, st>>>(tq, tk, tv, tg, a);
+        bwd_dq_kernel<64><<<grid_q, kBwdThreads, BwdSmem<64>::kTotal_dq, st>>>(tq, tk, tv, tg, to, a);
         bwd_dkv_kernel<64><<<grid_kv, kBwdThreads, BwdSmem<64>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
         bwd_combine_kernel<64><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     }
