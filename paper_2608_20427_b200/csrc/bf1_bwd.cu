@@ -31,6 +31,8 @@
 // M = 128 MMAs: tensor-memory lanes 64..127 then hold nothing of value and are not read.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "bf1_common.cuh"
 
 namespace bf1 {
@@ -65,6 +67,7 @@ struct BwdArgs {
     const int32_t* kv_count;
     const int32_t* kv_idx;
     const int32_t* num_qblocks;
+    const int32_t* order;      // may be null
     int32_t max_degree, capacity, total_tokens, hq, hkv, group;
     int32_t* status;
     float scale, scale_log2;
@@ -174,8 +177,8 @@ __device__ __forceinline__ void store_row_piece(uint32_t row_addr, int row, int 
 // One head per KV head: rows 64..127 of every column chunk of the Q and dO tiles are never written by a copy;
 // the MMAs still read them, so they are cleared once (they then give P = 0 and dS = 0 like rows past a sequence).
 template <int D>
-__device__ __forceinline__ void clear_idle_rows(uint32_t sQ, uint32_t sDO, int tid) {
-    for (int i = tid; i < 2 * (D / 64) * 512; i += kBwdThreads) {
+__device__ __forceinline__ void clear_idle_rows(uint32_t sQ, uint32_t sDO, int tid, int threads) {
+    for (int i = tid; i < 2 * (D / 64) * 512; i += threads) {
         const int which = i / ((D / 64) * 512), ch = (i / 512) % (D / 64), off = i % 512;
         st_shared_v4((which ? sDO : sQ) + ch * 16384 + 8192 + off * 16, 0u, 0u, 0u, 0u);
     }
@@ -198,66 +201,144 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t (&w)[4]) {
 }
 
 // ---- dQ --------------------------------------------------------------------------------------------------------
-
-// Warp roles of the two compute kernels: the row warps do the arithmetic on S and dP (one or two threads per tile
-// row), two warps issue copies (one thread keeps a TMA queue only about half full) and one issues MMAs.  Nobody
-// but the row warps ever waits for arithmetic, so copies and MMAs of the next list entry are under way while the
-// current one is being worked on.
-constexpr int kWarpLoadA = kRowWarps, kWarpLoadB = kRowWarps + 1, kWarpMma = kRowWarps + 2;
+//
+// One persistent CTA of 16 warps per SM.  Units (query block, KV head, pair of heads) are dealt out statically, in
+// the route's longest-list-first order KV head by KV head, back and forth over the CTAs so that each gets the same
+// mix.  Everything a unit needs travels through rings whose next entry is under way while the current one is in
+// use, across unit boundaries as well:
+//     warp 0    copies Q of every unit (two buffers) and the K tile of every list entry (ring of kStages)
+//     warp 1    copies dO of every unit, its O tile (into a whole ring stage, ahead of the unit's K/V tiles) and
+//               the V tiles
+//     warp 2    issues S and dP of every entry into one of two S/dP buffers in tensor memory, as soon as the K / V
+//               tiles are there and the dQ MMAs that read the buffer's last dS are done
+//     warp 3    issues the dQ MMAs of every entry; dQ accumulates in one of two buffers
+//     warps 4-7, 8-11   the arithmetic on S and dP, entries taken alternately by the two groups; dS (bf16) goes
+//               back into tensor memory over S, from where the dQ MMAs read it as their A operand
+//     warps 12-15   per unit: D_i = <dO_i, O_i> and the LSE of every row into shared memory (and D_i into the
+//               workspace, for the dK/dV kernel) one unit ahead; then the finished dQ tile of the unit before,
+//               from tensor memory to global memory
+// Every wait of a role is on a barrier it waits on once per phase, in phase order: a parity wait is only
+// meaningful one phase ahead.
+constexpr int kDqThreads = 512;
+constexpr int kStages = 3;
+// Q / dO buffer (and barrier) of unit n, and the parity of its n-th use
+__device__ __forceinline__ int qbuf(int n) { return n & 1; }
+__device__ __forceinline__ uint32_t qpar(int n) { return (n >> 1) & 1; }
 
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q,
-                                                             const __grid_constant__ CUtensorMap tm_k,
-                                                             const __grid_constant__ CUtensorMap tm_v,
-                                                             const __grid_constant__ CUtensorMap tm_do,
-                                                             const __grid_constant__ CUtensorMap tm_o,
-                                                             const BwdArgs a) {
-    using L = BwdSmem<D>;
+struct DqSmem {
+    static constexpr int kQBytes = 128 * D * 2;      // Q / dO / O tile [D / 64 chunks][128 rows][128 B]
+    static constexpr int kKVBytes = 64 * D * 2;      // K / V tile      [D / 64 chunks][64 rows][128 B]
+    static constexpr int kQ = 0;                     // [2]
+    static constexpr int kDO = kQ + 2 * kQBytes;     // [2]
+    static constexpr int kRing = kDO + 2 * kQBytes;  // [kStages] of K | V (or one O tile)
+    static constexpr int kRow = kRing + kStages * 2 * kKVBytes;   // D_i [2][128], LSE [2][128] (fp32)
+    static constexpr int kBar = kRow + 2048;
+    static constexpr int kUsed = kBar + 512;
+    // at least this much is requested so that a second CTA never fits an SM: each allocates all of tensor memory
+    static constexpr int kTotal = kUsed > 120 * 1024 ? kUsed : 120 * 1024;
+};
+
+struct DqUnit {
+    int ok, slot, kvh, pair, cnt, seq0, j, tok0, rows_valid;
+};
+
+// Unit n of this CTA (see above for the order).
+__device__ __forceinline__ DqUnit dq_unit(const BwdArgs& a, int n, int nqb, int pairs) {
+    DqUnit u;
+    const int per_head = nqb * pairs, total = per_head * a.hkv;
+    const int G = gridDim.x;
+    const int i = n * G + ((n & 1) ? G - 1 - (int)blockIdx.x : (int)blockIdx.x);
+    u.ok = i < total;
+    u.slot = u.kvh = u.pair = u.seq0 = u.j = u.tok0 = 0;
+    u.cnt = 1;
+    u.rows_valid = 0;
+    if (u.ok) {
+        u.kvh = i / per_head;
+        const int rem = i - u.kvh * per_head;
+        const int rank = rem / pairs;
+        u.pair = rem - rank * pairs;
+        int slot = a.order ? a.order[rank] : rank;
+        slot = min(max(slot, 0), nqb - 1);
+        u.slot = slot;
+        const int seq = a.qb_seq[slot];
+        u.j = a.qb_block[slot];
+        u.cnt = min(max(a.kv_count[slot], 1), a.max_degree);
+        u.seq0 = a.cu_seqlens[seq];
+        u.rows_valid = min(kBlock64, a.cu_seqlens[seq + 1] - u.seq0 - u.j * kBlock64);
+        u.tok0 = u.seq0 + u.j * kBlock64;
+    }
+    return u;
+}
+
+__device__ __forceinline__ void named_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                            const __grid_constant__ CUtensorMap tm_k,
+                                                            const __grid_constant__ CUtensorMap tm_v,
+                                                            const __grid_constant__ CUtensorMap tm_do,
+                                                            const __grid_constant__ CUtensorMap tm_o,
+                                                            const BwdArgs a) {
+    using L = DqSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
-    // no static shared memory: it would cost a whole extra kilobyte and with it the second CTA per SM
-    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_dq + 88);
-    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_dq + 92);
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar + 496);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar + 500);
+    float* s_drow = reinterpret_cast<float*>(smem + L::kRow);          // [2][128]
+    float* s_lse = s_drow + 256;                                       // [2][128]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int slot = blockIdx.x, kvh = blockIdx.y, pair = blockIdx.z;   // pair: which two query heads of the group
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
-    if (slot >= min(*a.num_qblocks, a.capacity)) return;
-    const int seq = a.qb_seq[slot], j = a.qb_block[slot];
-    const int cnt = min(max(a.kv_count[slot], 1), a.max_degree);
-    const int32_t* list = a.kv_idx + (size_t)slot * a.max_degree;
-    const int seq0 = a.cu_seqlens[seq];
-    const int seqlen = a.cu_seqlens[seq + 1] - seq0;
-    const int rows_valid = min(kBlock64, seqlen - j * kBlock64);
-    const int tok0 = seq0 + j * kBlock64;
+    const int nqb = min(*a.num_qblocks, a.capacity);
+    const int pairs = a.group == 4 ? 2 : 1;
 
     const uint32_t base = smem_u32(smem);
-    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sV = base + L::kV;
-    const uint32_t sO = sV;   // the O tile lies over V and the second K buffer until D_i has been computed
-    const uint32_t sKbuf[2] = {base + L::kK, base + L::kK1_dq};
-    // bar_q: Q, dO, O landed; bar_k[2], bar_v: a K / V tile landed; bar_sdp: S and dP computed; bar_ds: dS written
-    // (one arrival per row warp); bar_dq[2]: the dQ MMAs of an entry done (alternating, like the K buffers they
-    // free); bar_o: the O tile has been read (one arrival per row warp)
-    const uint32_t bar_q = base + L::kBar_dq, bar_k = bar_q + 8 /* [2] */, bar_v = bar_q + 24, bar_sdp = bar_q + 32,
-                   bar_ds = bar_q + 40, bar_dq = bar_q + 48 /* [2] */, bar_o = bar_q + 64;
+    const uint32_t bars = base + L::kBar;
+    // barriers (8 bytes each)
+    const uint32_t qdo_full = bars;                          // [2] Q and dO of a unit landed (both copy warps announce bytes)
+    const uint32_t qdo_free = qdo_full + 16;                 // [2] the unit's MMAs are done and its D_i computed
+    const uint32_t o_full = qdo_free + 16;                   // [2] the unit's O tile landed
+    const uint32_t row_full = o_full + 16;                   // [2] D_i and LSE of the unit's rows are in shared memory
+    const uint32_t row_free = row_full + 16;                 // [2] ... and have been read by both arithmetic groups (8 warps)
+    const uint32_t sdp_full = row_free + 16;                 // [2] S and dP of an entry computed
+    const uint32_t ds_ready = sdp_full + 16;                 // [2] dS written (4 warps)
+    const uint32_t dq_full = ds_ready + 16;                  // [2] the unit's dQ is complete
+    const uint32_t dq_free = dq_full + 16;                   // [2] ... and has been read out of tensor memory
+    const uint32_t dq_done = dq_free + 16;                   // [2] the dQ MMAs that read dS from an S / dP buffer are done
+    const uint32_t kv_full = dq_done + 16;                   // [kStages] a K and a V tile landed (both copy warps announce bytes)
+    const uint32_t ring_free = kv_full + 8 * kStages;        // [kStages] the stage's tiles (or O tile) have been used
+    static_assert(160 + 16 * kStages <= 496, "barriers overlap the words behind them");
     if (tid == 0) {
         s_abort = (base & 1023u) ? 1 : 0;
         if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
-        mbar_init(bar_q, 2);
-        mbar_init(bar_k, 1);
-        mbar_init(bar_k + 8, 1);
-        mbar_init(bar_v, 1);
-        mbar_init(bar_sdp, 1);
-        mbar_init(bar_ds, kRowWarps);
-        mbar_init(bar_dq, 1);
-        mbar_init(bar_dq + 8, 1);
-        mbar_init(bar_o, kRowWarps);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(qdo_full + 8 * b, 2);
+            mbar_init(qdo_free + 8 * b, 2);
+            mbar_init(o_full + 8 * b, 1);
+            mbar_init(row_full + 8 * b, 1);
+            mbar_init(row_free + 8 * b, 8);
+            mbar_init(sdp_full + 8 * b, 1);
+            mbar_init(ds_ready + 8 * b, 4);
+            mbar_init(dq_full + 8 * b, 1);
+            mbar_init(dq_free + 8 * b, 1);
+            mbar_init(dq_done + 8 * b, 1);
+        }
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(kv_full + 8 * s, 2);
+            mbar_init(ring_free + 8 * s, 1);
+        }
         fence_mbar_init();
     }
     __syncwarp();
     if (warp == 0) {
-        tmem_alloc(smem_u32(&s_tmem), 256);
+        tmem_alloc(smem_u32(&s_tmem), 512);
         tmem_relinquish();
     }
-    if (a.group == 1) clear_idle_rows<D>(sQ, sDO, tid);
+    if (a.group == 1) {   // one head per KV head: rows 64..127 of the Q / dO buffers are never written by a copy
+        clear_idle_rows<D>(base + L::kQ, base + L::kDO, tid, kDqThreads);
+        clear_idle_rows<D>(base + L::kQ + L::kQBytes, base + L::kDO + L::kQBytes, tid, kDqThreads);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -265,172 +346,241 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dq_kernel(const __grid_con
     volatile int* abort_flag = &s_abort;
     if (s_abort) {   // (uniform over the CTA)
         __syncthreads();
-        if (warp == 0) tmem_dealloc(tmem, 256);
+        if (warp == 0) tmem_dealloc(tmem, 512);
         return;
     }
-    // S and dP: 64 fp32 columns each; dS (bf16 pairs) takes over columns 0..15 and 32..47 of S; dQ: d columns
-    constexpr uint32_t kColS = 0, kColDP = 64, kColDQ = 128;
-    constexpr uint32_t kQTx = L::kQBytes;
-    const int head0 = kvh * a.group + pair * 2;
-    const uint32_t q_tx = a.group > 1 ? kQTx : kQTx / 2;   // one head per KV head: half a tile per copy set
+    // tensor memory: S | dP of buffer b at columns 128 b (dS takes over columns 0..15 and 32..47 of S), dQ of
+    // buffer b at 256 + 128 b
+    constexpr uint32_t kColDP = 64, kColDQ = 256;
+    const uint32_t q_tx = a.group > 1 ? L::kQBytes : L::kQBytes / 2;   // one head per KV head: half a tile per copy set
+    auto stage_k = [&](int s) { return base + L::kRing + s * 2 * L::kKVBytes; };
+    auto stage_v = [&](int s) { return base + L::kRing + s * 2 * L::kKVBytes + L::kKVBytes; };
 
-    if (warp == kWarpLoadA) {
-        // ---- copies, first half: dO, Q, then the K tiles (tile `it` in buffer it & 1, fetched two entries ahead) ----
-        const int p0 = list_entry(list, 0, cnt, j);
-        if (elect_one()) {
-            mbar_expect_tx(bar_q, 2 * q_tx);
-            load_q_tile<D>(sDO, &tm_do, tok0, head0, a.group, bar_q);
-            load_q_tile<D>(sQ, &tm_q, tok0, head0, a.group, bar_q);
-            mbar_expect_tx(bar_k, L::kKVBytes);
-            tma_load_4d(sKbuf[0], &tm_k, 0, seq0 + p0 * kBlock64, kvh, 0, bar_k);
-        }
-        __syncwarp();
-        if (cnt > 1) {
-            const int p1 = list_entry(list, 1, cnt, j);
-            mbar_wait(bar_o, 0, abort_flag, a.status);
+    if (warp == 0 || warp == 1) {
+        // ---- copies ----
+        const bool first = warp == 0;
+        int r = 0;                      // ring entries so far: stage r % kStages, its phase r / kStages
+        int rs = 0, rk = 0;             // the same as (stage, phase counter)
+        auto ring_wait_free = [&]() {
+            if (r >= kStages) mbar_wait(ring_free + 8 * rs, (rk - 1) & 1, abort_flag, a.status);
+        };
+        auto ring_next = [&]() {
+            ++r;
+            if (++rs == kStages) { rs = 0; ++rk; }
+        };
+        DqUnit u = dq_unit(a, 0, nqb, pairs);
+        for (int n = 0; u.ok; ++n) {
+            const DqUnit un = dq_unit(a, n + 1, nqb, pairs);
+            const int b = n & 1, head0 = u.kvh * a.group + u.pair * 2;
+            const int32_t* list = a.kv_idx + (size_t)u.slot * a.max_degree;
+            const int qb = qbuf(n);
+            if (n >= 2) mbar_wait(qdo_free + 8 * qb, qpar(n - 2), abort_flag, a.status);
             if (elect_one()) {
-                mbar_expect_tx(bar_k + 8, L::kKVBytes);
-                tma_load_4d(sKbuf[1], &tm_k, 0, seq0 + p1 * kBlock64, kvh, 0, bar_k + 8);
+                mbar_expect_tx(qdo_full + 8 * qb, q_tx);
+                if (first) load_q_tile<D>(base + L::kQ + qb * L::kQBytes, &tm_q, u.tok0, head0, a.group, qdo_full + 8 * qb);
+                else load_q_tile<D>(base + L::kDO + qb * L::kQBytes, &tm_do, u.tok0, head0, a.group, qdo_full + 8 * qb);
             }
             __syncwarp();
-        }
-        for (int it = 0; it + 2 < cnt; ++it) {
-            const int p = list_entry(list, it + 2, cnt, j);
-            mbar_wait(bar_dq + 8 * (it & 1), (it >> 1) & 1, abort_flag, a.status);   // dQ(it) done: its K buffer is free
-            if (elect_one()) {
-                mbar_expect_tx(bar_k + 8 * (it & 1), L::kKVBytes);
-                tma_load_4d(sKbuf[it & 1], &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_k + 8 * (it & 1));
+            // the O tile's ring entry
+            if (!first) {
+                ring_wait_free();
+                if (elect_one()) {
+                    mbar_expect_tx(o_full + 8 * b, q_tx);
+                    load_q_tile<D>(stage_k(rs), &tm_o, u.tok0, head0, a.group, o_full + 8 * b);
+                }
+                __syncwarp();
             }
-            __syncwarp();
-        }
-    } else if (warp == kWarpLoadB) {
-        // ---- copies, second half: O, then the V tiles (one buffer, refetched as soon as dP has been computed) ----
-        if (elect_one()) {
-            mbar_expect_tx(bar_q, q_tx);
-            load_q_tile<D>(sO, &tm_o, tok0, head0, a.group, bar_q);
-        }
-        __syncwarp();
-        for (int it = 0; it < cnt; ++it) {
-            const int p = list_entry(list, it, cnt, j);
-            if (it == 0) mbar_wait(bar_o, 0, abort_flag, a.status);
-            else mbar_wait(bar_sdp, (it - 1) & 1, abort_flag, a.status);
-            if (elect_one()) {
-                mbar_expect_tx(bar_v, L::kKVBytes);
-                tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_v);
+            ring_next();
+            for (int it = 0; it < u.cnt; ++it) {
+                const int p = list_entry(list, it, u.cnt, u.j);
+                ring_wait_free();
+                if (elect_one()) {
+                    mbar_expect_tx(kv_full + 8 * rs, L::kKVBytes);
+                    if (first) tma_load_4d(stage_k(rs), &tm_k, 0, u.seq0 + p * kBlock64, u.kvh, 0, kv_full + 8 * rs);
+                    else tma_load_4d(stage_v(rs), &tm_v, 0, u.seq0 + p * kBlock64, u.kvh, 0, kv_full + 8 * rs);
+                }
+                __syncwarp();
+                ring_next();
             }
-            __syncwarp();
+            u = un;
         }
-    } else if (warp == kWarpMma) {
-        // ---- MMAs: S, dP of entry it + 1 are issued right behind dQ of entry it (the pipe runs them in order, so the
-        // new S only overwrites dS once the dQ MMAs have read it) ----
+    } else if (warp == 2 || warp == 3) {
+        // ---- MMAs: warp 2 issues S and dP of every entry, warp 3 its dQ.  Two warps, because what surrounds a batch of
+        // MMAs (barrier round trips through shared memory, the unit bookkeeping) costs several hundred cycles per
+        // entry, during which a single issuing warp would leave the pipe empty. ----
         constexpr uint32_t kHi = desc_hi_sw128(1024);
         constexpr uint32_t kIdQ = idesc_bf16_f32(D, true);             // dQ: 128 x d, A from tensor memory, B (K tile) MN-major
-        mbar_wait(bar_q, 0, abort_flag, a.status);
-        for (int it = 0; it < cnt; ++it) {
-            const int kb = it & 1;
-            mbar_wait(bar_k + 8 * kb, (it >> 1) & 1, abort_flag, a.status);
-            mbar_wait(bar_v, it & 1, abort_flag, a.status);
-            tc_fence_after();
-            if (elect_one()) {
-                issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sKbuf[kb], sV);
-                mma_commit(bar_sdp);
-            }
-            __syncwarp();
-            mbar_wait(bar_ds, it & 1, abort_flag, a.status);
-            tc_fence_after();
-            if (elect_one()) {
-                // dQ += dS K: A = dS [128 q][64 kv] from tensor memory (16 kv = 8 columns per step; keys 0..31 sit in
-                // columns 0..15, keys 32..63 in columns 32..47), B = K tile MN-major (16 kv rows = 2048 bytes per step,
-                // next 64 d columns 8 KB away)
+        DqUnit u = dq_unit(a, 0, nqb, pairs);
+        int t = 0, rs = 1 % kStages;       // entries so far; ring stage of the entry (entry 0 of the ring is unit 0's O tile)
+        uint32_t kv_phase = 0;             // per stage: parity of the K / V tiles put into it so far
+        for (int n = 0; u.ok; ++n) {
+            const DqUnit un = dq_unit(a, n + 1, nqb, pairs);
+            const int b = n & 1;
+            if (warp == 2) mbar_wait(qdo_full + 8 * b, qpar(n), abort_flag, a.status);
+            else if (n >= 2) mbar_wait(dq_free + 8 * b, qpar(n - 2), abort_flag, a.status);
+            for (int it = 0; it < u.cnt; ++it) {
+                const int sb = t & 1;
+                if (warp == 2) {
+                    // the buffer's last dS must have been read by its dQ MMAs before S overwrites it
+                    if (t >= 2) mbar_wait(dq_done + 8 * sb, ((t >> 1) - 1) & 1, abort_flag, a.status);
+                    mbar_wait(kv_full + 8 * rs, (kv_phase >> rs) & 1, abort_flag, a.status);
+                    tc_fence_after();
+                    if (elect_one()) {
+                        issue_s_dp<D>(tmem + sb * 128, tmem + sb * 128 + kColDP, base + L::kQ + b * L::kQBytes,
+                                      base + L::kDO + b * L::kQBytes, stage_k(rs), stage_v(rs));
+                        mma_commit(sdp_full + 8 * sb);
+                    }
+                    __syncwarp();
+                } else {
+                    mbar_wait(ds_ready + 8 * sb, (t >> 1) & 1, abort_flag, a.status);
+                    tc_fence_after();
+                    if (elect_one()) {
+                        // dQ += dS K: A = dS [128 q][64 kv] from tensor memory (16 kv = 8 columns per step; keys 0..31 sit in
+                        // columns 0..15, keys 32..63 in columns 32..47), B = K tile MN-major (16 kv rows = 2048 bytes per step,
+                        // next 64 d columns 8 KB away)
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {   // 64 kv rows in steps of 16
-                    const uint32_t blo = desc_lo_sw128(sKbuf[kb], 8192) + ((kk * 2048) >> 4);
-                    const uint32_t a_ds = tmem + kColS + (kk >> 1) * 32 + (kk & 1) * 8;
-                    if (it == 0 && kk == 0) mma_ts_lohi<false>(tmem + kColDQ, a_ds, blo, kHi, kIdQ);
-                    else mma_ts_lohi<true>(tmem + kColDQ, a_ds, blo, kHi, kIdQ);
+                        for (int kk = 0; kk < 4; ++kk) {   // 64 kv rows in steps of 16
+                            const uint32_t blo = desc_lo_sw128(stage_k(rs), 8192) + ((kk * 2048) >> 4);
+                            const uint32_t a_ds = tmem + sb * 128 + (kk >> 1) * 32 + (kk & 1) * 8;
+                            if (kk == 0) {
+                                if (it == 0) mma_ts_lohi<false>(tmem + kColDQ + b * 128, a_ds, blo, kHi, kIdQ);
+                                else mma_ts_lohi<true>(tmem + kColDQ + b * 128, a_ds, blo, kHi, kIdQ);
+                            } else {
+                                mma_ts_lohi<true>(tmem + kColDQ + b * 128, a_ds, blo, kHi, kIdQ);
+                            }
+                        }
+                        mma_commit(dq_done + 8 * sb);
+                        mma_commit(ring_free + 8 * rs);
+                        if (it == u.cnt - 1) {
+                            mma_commit(dq_full + 8 * b);
+                            mma_commit(qdo_free + 8 * b);
+                        }
+                    }
+                    __syncwarp();
                 }
-                mma_commit(bar_dq + 8 * kb);
+                kv_phase ^= 1u << rs;
+                ++t;
+                if (++rs == kStages) rs = 0;
             }
-            __syncwarp();
+            if (++rs == kStages) rs = 0;   // the next unit's O tile
+            u = un;
         }
-    } else {
-        // ---- row warps: tile row (head hl, token tl of the query block) and which half of a tile's 64 key columns ----
-        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        const int row = tid & 127, half = tid >> 7;
-        const int hl = row >> 6, tl = row & 63;
-        const int h = head0 + hl;
-        const int tok = tok0 + tl;
-        const bool row_ok = tl < rows_valid && pair * 2 + hl < a.group;   // G = 1: rows 64..127 belong to no head
-        // D_i = <dO_i, O_i> from the two tiles in shared memory (both threads of a row compute it), and the row's
-        // LSE in the log2 domain
-        float lse2 = INFINITY;
-        if (row_ok) lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
-        mbar_wait(bar_q, 0, abort_flag, a.status);
-        float Drow = 0.f;
-        if (row_ok) {
-#pragma unroll
-            for (int c = 0; c < D / 8; ++c) {   // 16-byte pieces of the row: chunk c / 8 of 64 columns, piece c % 8
-                const uint32_t off = (c >> 3) * 16384 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
-                uint32_t ow[4], gw[4];
-                ld_shared_v4(sO + off, ow);
-                ld_shared_v4(sDO + off, gw);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    Drow = fmaf(__uint_as_float(ow[e] << 16), __uint_as_float(gw[e] << 16), Drow);
-                    Drow = fmaf(__uint_as_float(ow[e] & 0xffff0000u), __uint_as_float(gw[e] & 0xffff0000u), Drow);
+    } else if (warp >= 4 && warp < 12) {
+        // ---- arithmetic on S and dP: this thread's tile row (head hl, token tl) in group g's entries ----
+        const int g = (warp - 4) >> 2;
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + g * 128;
+        const int row = tid & 127, tl = row & 63;
+        int t = 0;
+        DqUnit u = dq_unit(a, 0, nqb, pairs);
+        for (int n = 0; u.ok; ++n) {
+            const DqUnit un = dq_unit(a, n + 1, nqb, pairs);
+            const int b = n & 1;
+            mbar_wait(row_full + 8 * b, (n >> 1) & 1, abort_flag, a.status);
+            const float Drow = s_drow[b * 128 + row], lse2 = s_lse[b * 128 + row];
+            for (int it = (t & 1) == g ? 0 : 1; it < u.cnt; it += 2) {
+                const int tt = t + it;
+                mbar_wait(sdp_full + 8 * g, (tt >> 1) & 1, abort_flag, a.status);
+                tc_fence_after();
+#pragma unroll 1
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t pw[16], dw[16];
+                    p_and_ds(t_lane, t_lane + kColDP, hh, tl, it == u.cnt - 1, lse2, Drow, a.scale, a.scale_log2, pw, dw);
+                    // dS as the A operand of the dQ MMAs: bf16 pairs, written over the first 16 of the 32 S columns just read
+                    tmem_st16(t_lane + hh * 32, dw);
                 }
-            }
-            if (half == 0) a.delta[(size_t)h * a.total_tokens + tok] = Drow;   // for the dK/dV kernel
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_o);
-
-        for (int it = 0; it < cnt; ++it) {
-            const bool diag = (it == cnt - 1);
-            mbar_wait(bar_sdp, it & 1, abort_flag, a.status);
-            tc_fence_after();
-            for (int hh = half * (2 / kPerRow); hh < (half + 1) * (2 / kPerRow); ++hh) {
-                uint32_t pw[16], dw[16];
-                p_and_ds(t_lane + kColS, t_lane + kColDP, hh, tl, diag, lse2, Drow, a.scale, a.scale_log2, pw, dw);
-                // dS as the A operand of the next MMA: bf16 pairs, written over the first 16 of the 32 S columns this
-                // thread has just read (its own columns only: the row's other thread may still be reading its half)
+                tmem_wait_st();
+                tc_fence_before();
                 __syncwarp();
-                tmem_st16(t_lane + kColS + hh * 32, dw);
+                if (lane == 0) mbar_arrive(ds_ready + 8 * g);
             }
-            tmem_wait_st();
-            tc_fence_before();
+            t += u.cnt;
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_ds);
+            if (lane == 0) mbar_arrive(row_free + 8 * b);
+            u = un;
         }
-        // the last dQ MMA
-        mbar_wait(bar_dq + 8 * ((cnt - 1) & 1), ((cnt - 1) >> 1) & 1, abort_flag, a.status);
-        tc_fence_after();
-
-        // ---- dQ rows: each of a row's threads stores its share of the columns ----
-        constexpr int kColsPerThread = D / kPerRow;
-        __nv_bfloat16* dqrow = a.dq + ((size_t)tok * a.hq + h) * D + half * kColsPerThread;
-#pragma unroll
-        for (int c = 0; c < kColsPerThread / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(t_lane + kColDQ + half * kColsPerThread + c * 32, r);
-            tmem_wait_ld();
+    } else if (warp >= 12) {
+        // ---- per unit: D_i and LSE one unit ahead; the finished dQ tile of the unit before ----
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const int row = tid & 127, hl = row >> 6, tl = row & 63;
+        int r = 0;   // ring entry of the current unit's O tile
+        auto prologue = [&](const DqUnit& u, int n) {
+            const int b = n & 1;
+            const int h = u.kvh * a.group + u.pair * 2 + hl, tok = u.tok0 + tl;
+            const bool row_ok = tl < u.rows_valid && u.pair * 2 + hl < a.group;   // G = 1: rows 64..127 belong to no head
+            float lse2 = INFINITY, Drow = 0.f;
+            if (row_ok) lse2 = a.lse[(size_t)h * a.total_tokens + tok] * 1.4426950408889634f;
+            mbar_wait(qdo_full + 8 * qbuf(n), qpar(n), abort_flag, a.status);
+            mbar_wait(o_full + 8 * b, (n >> 1) & 1, abort_flag, a.status);
+            if (n >= 2) mbar_wait(row_free + 8 * b, ((n >> 1) - 1) & 1, abort_flag, a.status);
+            const int rs = r % kStages;
             if (row_ok) {
+                const uint32_t sO = stage_k(rs), sDO = base + L::kDO + qbuf(n) * L::kQBytes;
 #pragma unroll
-                for (int e = 0; e < 32; e += 8) {
-                    uint4 w;
-                    w.x = pack_bf16x2(__uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
-                    w.y = pack_bf16x2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                    w.z = pack_bf16x2(__uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
-                    w.w = pack_bf16x2(__uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
-                    *reinterpret_cast<uint4*>(dqrow + c * 32 + e) = w;
+                for (int c = 0; c < D / 8; ++c) {   // 16-byte pieces of the row: chunk c / 8 of 64 columns, piece c % 8
+                    const uint32_t off = (c >> 3) * 16384 + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                    uint32_t ow[4], gw[4];
+                    ld_shared_v4(sO + off, ow);
+                    ld_shared_v4(sDO + off, gw);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        Drow = fmaf(__uint_as_float(ow[e] << 16), __uint_as_float(gw[e] << 16), Drow);
+                        Drow = fmaf(__uint_as_float(ow[e] & 0xffff0000u), __uint_as_float(gw[e] & 0xffff0000u), Drow);
+                    }
+                }
+                a.delta[(size_t)h * a.total_tokens + tok] = Drow;   // for the dK/dV kernel
+            }
+            s_drow[b * 128 + row] = Drow;
+            s_lse[b * 128 + row] = lse2;
+            named_sync(1, 128);
+            if ((tid & 127) == 0) {
+                mbar_arrive(ring_free + 8 * rs);
+                mbar_arrive(qdo_free + 8 * qbuf(n));
+                mbar_arrive(row_full + 8 * b);
+            }
+            r += u.cnt + 1;
+        };
+        DqUnit u = dq_unit(a, 0, nqb, pairs);
+        if (u.ok) prologue(u, 0);
+        for (int n = 0; u.ok; ++n) {
+            const DqUnit un = dq_unit(a, n + 1, nqb, pairs);
+            if (un.ok) prologue(un, n + 1);
+            const int b = n & 1;
+            const int h = u.kvh * a.group + u.pair * 2 + hl, tok = u.tok0 + tl;
+            const bool row_ok = tl < u.rows_valid && u.pair * 2 + hl < a.group;
+            mbar_wait(dq_full + 8 * b, (n >> 1) & 1, abort_flag, a.status);
+            tc_fence_after();
+            __nv_bfloat16* dqrow = a.dq + ((size_t)tok * a.hq + h) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(t_lane + kColDQ + b * 128 + c * 32, v);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(v[e + 0]), __uint_as_float(v[e + 1]));
+                        w.y = pack_bf16x2(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                        w.z = pack_bf16x2(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+                        w.w = pack_bf16x2(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
+                        *reinterpret_cast<uint4*>(dqrow + c * 32 + e) = w;
+                    }
                 }
             }
+            tc_fence_before();
+            named_sync(1, 128);
+            if ((tid & 127) == 0) mbar_arrive(dq_free + 8 * b);
+            u = un;
         }
-        tc_fence_before();
     }
+    tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 256);
+    if (warp == 0) tmem_dealloc(tmem, 512);
 }
+
+// Warp roles of the dK/dV kernel: the row warps do the arithmetic on S and dP, two warps issue copies (one thread
+// keeps a TMA queue only about half full) and one issues MMAs.
+constexpr int kWarpLoadA = kRowWarps, kWarpLoadB = kRowWarps + 1, kWarpMma = kRowWarps + 2;
 
 // ---- the inverse route -----------------------------------------------------------------------------------------
 
@@ -611,7 +761,7 @@ __global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_co
         tmem_alloc(smem_u32(&s_tmem), 256);
         tmem_relinquish();
     }
-    if (a.group == 1) clear_idle_rows<D>(sQ, sDO, tid);
+    if (a.group == 1) clear_idle_rows<D>(sQ, sDO, tid, kBwdThreads);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -846,8 +996,8 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     if (dev < 0 || dev >= 64) return fail(BF1_ERR_NO_DEVICE, "device ordinal %d out of range", dev);
     if (!configured[dev]) {
         // two CTAs per SM need the whole shared-memory carve-out
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal_dq));
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal_dq));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<128>::kTotal));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<64>::kTotal));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal_kv));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal_kv));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
@@ -874,6 +1024,7 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.kv_count = route->kv_count;
     a.kv_idx = route->kv_idx;
     a.num_qblocks = route->num_qblocks;
+    a.order = route->order;
     a.max_degree = route->max_degree;
     a.capacity = cap;
     a.total_tokens = (int32_t)total_tokens;
@@ -912,14 +1063,16 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     inverse_route_kernel<true><<<cap, 256, 0, st>>>(a);
     BF1_CUDA_CHECK(cudaGetLastError());
     // ... dQ (and D_i) along the route, dK / dV along its inverse
-    dim3 grid_q(cap, hkv, group == 4 ? 2 : 1);   // z: pairs of query heads
+    int sms = 0;
+    BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int grid_q = (int)std::min<int64_t>(sms, (int64_t)cap * hkv * (group == 4 ? 2 : 1));   // persistent: one CTA per SM
     dim3 grid_kv((unsigned)lay.n_units, hkv);
     if (d == 128) {
-        bwd_dq_kernel<128><<<grid_q, kBwdThreads, BwdSmem<128>::kTotal_dq, st>>>(tq, tk, tv, tg, to, a);
+        bwd_dq_kernel<128><<<grid_q, kDqThreads, DqSmem<128>::kTotal, st>>>(tq, tk, tv, tg, to, a);
         bwd_dkv_kernel<128><<<grid_kv, kBwdThreads, BwdSmem<128>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
         bwd_combine_kernel<128><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     } else {
-        bwd_dq_kernel<64><<<grid_q, kBwdThreads, BwdSmem<64>::kTotal_dq, st>>>(tq, tk, tv, tg, to, a);
+        bwd_dq_kernel<64><<<grid_q, kDqThreads, DqSmem<64>::kTotal, st>>>(tq, tk, tv, tg, to, a);
         bwd_dkv_kernel<64><<<grid_kv, kBwdThreads, BwdSmem<64>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
         bwd_combine_kernel<64><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     }
