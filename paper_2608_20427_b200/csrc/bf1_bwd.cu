@@ -212,8 +212,8 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t (&w)[4]) {
 //     warp 2    issues S and dP of every entry into one of two S/dP buffers in tensor memory, as soon as the K / V
 //               tiles are there and the dQ MMAs that read the buffer's last dS are done
 //     warp 3    issues the dQ MMAs of every entry; dQ accumulates in one of two buffers
-//     warps 4-7, 8-11   the arithmetic on S and dP, entries taken alternately by the two groups; dS (bf16) goes
-//               back into tensor memory over S, from where the dQ MMAs read it as their A operand
+//     warps 4-11   the arithmetic on S and dP, two threads per tile row (32 key columns each); dS (bf16) goes back
+//               into tensor memory over S, from where the dQ MMAs read it as their A operand
 //     warps 12-15   per unit: D_i = <dO_i, O_i> and the LSE of every row into shared memory (and D_i into the
 //               workspace, for the dK/dV kernel) one unit ahead; then the finished dQ tile of the unit before,
 //               from tensor memory to global memory
@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
     const uint32_t row_full = o_full + 16;                   // [2] D_i and LSE of the unit's rows are in shared memory
     const uint32_t row_free = row_full + 16;                 // [2] ... and have been read by both arithmetic groups (8 warps)
     const uint32_t sdp_full = row_free + 16;                 // [2] S and dP of an entry computed
-    const uint32_t ds_ready = sdp_full + 16;                 // [2] dS written (4 warps)
+    const uint32_t ds_ready = sdp_full + 16;                 // [2] dS written (8 warps)
     const uint32_t dq_full = ds_ready + 16;                  // [2] the unit's dQ is complete
     const uint32_t dq_free = dq_full + 16;                   // [2] ... and has been read out of tensor memory
     const uint32_t dq_done = dq_free + 16;                   // [2] the dQ MMAs that read dS from an S / dP buffer are done
@@ -319,7 +319,7 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
             mbar_init(row_full + 8 * b, 1);
             mbar_init(row_free + 8 * b, 8);
             mbar_init(sdp_full + 8 * b, 1);
-            mbar_init(ds_ready + 8 * b, 4);
+            mbar_init(ds_ready + 8 * b, 8);
             mbar_init(dq_full + 8 * b, 1);
             mbar_init(dq_free + 8 * b, 1);
             mbar_init(dq_done + 8 * b, 1);
@@ -466,9 +466,10 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
             u = un;
         }
     } else if (warp >= 4 && warp < 12) {
-        // ---- arithmetic on S and dP: this thread's tile row (head hl, token tl) in group g's entries ----
-        const int g = (warp - 4) >> 2;
-        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + g * 128;
+        // ---- arithmetic on S and dP: two threads per tile row (head hl, token tl), warps 4-7 on key columns 0..31 and
+        // warps 8-11 on columns 32..63 of every entry ----
+        const int half = (warp - 4) >> 2;
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const int row = tid & 127, tl = row & 63;
         int t = 0;
         DqUnit u = dq_unit(a, 0, nqb, pairs);
@@ -477,23 +478,19 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
             const int b = n & 1;
             mbar_wait(row_full + 8 * b, (n >> 1) & 1, abort_flag, a.status);
             const float Drow = s_drow[b * 128 + row], lse2 = s_lse[b * 128 + row];
-            for (int it = (t & 1) == g ? 0 : 1; it < u.cnt; it += 2) {
-                const int tt = t + it;
-                mbar_wait(sdp_full + 8 * g, (tt >> 1) & 1, abort_flag, a.status);
+            for (int it = 0; it < u.cnt; ++it, ++t) {
+                const int sb = t & 1;
+                mbar_wait(sdp_full + 8 * sb, (t >> 1) & 1, abort_flag, a.status);
                 tc_fence_after();
-#pragma unroll 1
-                for (int hh = 0; hh < 2; ++hh) {
-                    uint32_t pw[16], dw[16];
-                    p_and_ds(t_lane, t_lane + kColDP, hh, tl, it == u.cnt - 1, lse2, Drow, a.scale, a.scale_log2, pw, dw);
-                    // dS as the A operand of the dQ MMAs: bf16 pairs, written over the first 16 of the 32 S columns just read
-                    tmem_st16(t_lane + hh * 32, dw);
-                }
+                uint32_t pw[16], dw[16];
+                p_and_ds(t_lane + sb * 128, t_lane + sb * 128 + kColDP, half, tl, it == u.cnt - 1, lse2, Drow, a.scale, a.scale_log2, pw, dw);
+                // dS as the A operand of the dQ MMAs: bf16 pairs, written over the first 16 of the 32 S columns just read
+                tmem_st16(t_lane + sb * 128 + half * 32, dw);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(ds_ready + 8 * g);
+                if (lane == 0) mbar_arrive(ds_ready + 8 * sb);
             }
-            t += u.cnt;
             __syncwarp();
             if (lane == 0) mbar_arrive(row_free + 8 * b);
             u = un;
