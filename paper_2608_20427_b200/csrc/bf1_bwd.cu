@@ -38,10 +38,6 @@
 namespace bf1 {
 
 constexpr int kBlock64 = 64;     // b: tokens per block
-constexpr int kRowThreads = 128;               // threads that work on a tile's 128 rows
-constexpr int kPerRow = kRowThreads / 128;     // two per row: each takes 32 of a tile's 64 key columns
-constexpr int kRowWarps = kRowThreads / 32;
-constexpr int kBwdThreads = kRowThreads + 96;  // + two copy warps and one MMA warp
 constexpr int kMinChunk = 16;    // readers per dK/dV unit, at least
 
 // The inverse route and the units of bwd_dkv_kernel, all inside the caller's workspace.
@@ -90,31 +86,9 @@ __device__ __forceinline__ int list_entry(const int32_t* list, int e, int cnt, i
     return p;
 }
 
-template <int D>
-struct BwdSmem {
-    static constexpr int kQBytes = 128 * D * 2;      // Q / dO tile [D / 64 chunks][128 rows][128 B]
-    static constexpr int kKVBytes = 64 * D * 2;      // K / V tile  [D / 64 chunks][64 rows][128 B]
-    static constexpr int kQ = 0;
-    static constexpr int kDO = kQ + kQBytes;
-    static constexpr int kK = kDO + kQBytes;
-    static constexpr int kV = kK + kKVBytes;
-    // dQ kernel: dS goes to tensor memory, not to shared memory; the room it leaves is a second K buffer, so that
-    // the next K tile travels while the current one is in use (V is only needed for dP and is refetched early).
-    static constexpr int kK1_dq = kV + kKVBytes;
-    static constexpr int kBar_dq = kK1_dq + kKVBytes;
-    static constexpr int kTotal_dq = kBar_dq + 96;
-    // dK/dV kernel: P and dS [128 q rows][64 kv] bf16, 128-byte rows, swizzled (16 KB each).  At d = 128, P takes
-    // over V's buffer and dS takes over K's once S and dP have been computed (K and V are fetched again for the
-    // next reader; they come from L2); at d = 64 the K / V tiles are only 8 KB, so P and dS get room of their own.
-    static constexpr int kP_kv = D == 128 ? kV : kV + kKVBytes;
-    static constexpr int kDS_kv = D == 128 ? kK : kP_kv + 16384;
-    static constexpr int kBar_kv = D == 128 ? kV + kKVBytes : kDS_kv + 16384;
-    static constexpr int kTotal_kv = kBar_kv + 64;
-};
-
 // ---- pieces shared by the two compute kernels ------------------------------------------------------------------
 
-// S = Q K^T and dP = dO V^T: D / 16 k-steps over the head dimension (thread 0 only).
+// S = Q K^T and dP = dO V^T: D / 16 k-steps over the head dimension (one thread).
 template <int D>
 __device__ __forceinline__ void issue_s_dp(uint32_t t_s, uint32_t t_dp, uint32_t sQ, uint32_t sDO, uint32_t sK, uint32_t sV) {
     constexpr uint32_t kHi = desc_hi_sw128(1024);
@@ -575,10 +549,6 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-// Warp roles of the dK/dV kernel: the row warps do the arithmetic on S and dP, two warps issue copies (one thread
-// keeps a TMA queue only about half full) and one issues MMAs.
-constexpr int kWarpLoadA = kRowWarps, kWarpLoadB = kRowWarps + 1, kWarpMma = kRowWarps + 2;
-
 // ---- the inverse route -----------------------------------------------------------------------------------------
 
 // One CTA per KV slot: its readers are the query slots g >= it of the same sequence whose list names its block
@@ -714,191 +684,317 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
 }
 
 // ---- dK, dV ----------------------------------------------------------------------------------------------------
+//
+// One persistent CTA of 16 warps per SM.  A unit is (KV block, KV head, run of the block's readers); units are
+// dealt out statically KV head by KV head, back and forth over the CTAs.  K and V of a unit stay in shared memory
+// (two buffers: the next unit's arrive early), Q and dO of every step (a reader and a pair of its heads) travel
+// through a ring of two stages:
+//     warp 0    copies K of every unit and Q of every step;  warp 1: V and dO
+//     warp 2    issues S = Q K^T and dP = dO V^T of every step into one of two S/dP buffers in tensor memory
+//     warp 3    issues dV^T += dO^T P and dK^T += Q^T dS of every step; the sums stay in one of two accumulator
+//               buffers in tensor memory across all steps of the unit
+//     warps 4-11   the arithmetic on S and dP (two threads per tile row), P and dS as bf16 tiles to shared memory
+//     warps 12-15  the finished sums of the unit before, from tensor memory to global memory
+constexpr int kDkvThreads = 512;
 
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 2) bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q,
+struct DkvSmem {
+    static constexpr int kQBytes = 128 * D * 2;      // Q / dO tile [D / 64 chunks][128 rows][128 B]
+    static constexpr int kKVBytes = 64 * D * 2;      // K / V tile  [D / 64 chunks][64 rows][128 B]
+    static constexpr int kQ = 0;                     // [2]
+    static constexpr int kDO = kQ + 2 * kQBytes;     // [2]
+    static constexpr int kK = kDO + 2 * kQBytes;     // [2]
+    static constexpr int kV = kK + 2 * kKVBytes;     // [2]
+    static constexpr int kP = kV + 2 * kKVBytes;     // P  [128 q rows][64 kv] bf16, 128-byte rows, swizzled
+    static constexpr int kDS = kP + 16384;           // dS likewise
+    static constexpr int kBar = kDS + 16384;
+    static constexpr int kUsed = kBar + 512;
+    // at least this much is requested so that a second CTA never fits an SM: each allocates all of tensor memory
+    static constexpr int kTotal = kUsed > 120 * 1024 ? kUsed : 120 * 1024;
+};
+
+struct DkvUnit {
+    int ok, gp, kvh, r_begin, steps, part, seq0, seqlen, p, kv_valid;
+};
+
+// Unit n of this CTA.
+__device__ __forceinline__ DkvUnit dkv_unit(const BwdArgs& a, int n, int n_units, int pairs) {
+    DkvUnit u;
+    const int total = n_units * a.hkv;
+    const int G = gridDim.x;
+    const int i = n * G + ((n & 1) ? G - 1 - (int)blockIdx.x : (int)blockIdx.x);
+    u.ok = i < total;
+    u.gp = u.kvh = u.r_begin = u.seq0 = u.seqlen = u.p = u.kv_valid = 0;
+    u.steps = 0;
+    u.part = -1;
+    if (u.ok) {
+        u.kvh = i / n_units;
+        const int unit = i - u.kvh * n_units;
+        u.gp = a.inv.unit_slot[unit];
+        u.r_begin = a.inv.unit_begin[unit];
+        u.steps = (a.inv.unit_end[unit] - u.r_begin) * pairs;
+        u.part = a.inv.unit_part[unit];
+        const int seq = a.qb_seq[u.gp];
+        u.p = a.qb_block[u.gp];
+        u.seq0 = a.cu_seqlens[seq];
+        u.seqlen = a.cu_seqlens[seq + 1] - u.seq0;
+        u.kv_valid = min(kBlock64, u.seqlen - u.p * kBlock64);      // key rows of this block inside the sequence
+    }
+    return u;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                               const __grid_constant__ CUtensorMap tm_k,
                                                               const __grid_constant__ CUtensorMap tm_v,
                                                               const __grid_constant__ CUtensorMap tm_do,
                                                               const BwdArgs a) {
-    using L = BwdSmem<D>;
+    using L = DkvSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar_kv + 48);
-    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar_kv + 52);
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + L::kBar + 496);
+    int& s_abort = *reinterpret_cast<int*>(smem + L::kBar + 500);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int unit = blockIdx.x, kvh = blockIdx.y;
     if (a.status && (*a.status & BF1_DEV_WAIT_TIMEOUT)) return;
-    if (unit >= a.inv.scalars[0]) return;
-    const int gp = a.inv.unit_slot[unit];
-    const int r_begin = a.inv.unit_begin[unit], r_end = a.inv.unit_end[unit], part = a.inv.unit_part[unit];
-    const int seq = a.qb_seq[gp], p = a.qb_block[gp];
-    const int seq0 = a.cu_seqlens[seq];
-    const int seqlen = a.cu_seqlens[seq + 1] - seq0;
-    const int kv_valid = min(kBlock64, seqlen - p * kBlock64);      // key rows of this block inside the sequence
+    const int n_units = a.inv.scalars[0];
     const int pairs = a.group == 4 ? 2 : 1;
 
     const uint32_t base = smem_u32(smem);
-    const uint32_t sQ = base + L::kQ, sDO = base + L::kDO, sK = base + L::kK, sV = base + L::kV;
-    const uint32_t sP = base + L::kP_kv, sDS = base + L::kDS_kv;
-    // bar_ld: the four tiles of a step landed (both copy warps announce their bytes); bar_sdp: S and dP computed;
-    // bar_pds: P and dS written (one arrival per row warp); bar_acc: the step's dV^T / dK^T MMAs done, every buffer
-    // is free again
-    const uint32_t bar_ld = base + L::kBar_kv, bar_sdp = bar_ld + 8, bar_pds = bar_ld + 16, bar_acc = bar_ld + 24;
+    const uint32_t bars = base + L::kBar;
+    const uint32_t kv_full = bars;                 // [2] K and V of a unit landed (both copy warps announce bytes)
+    const uint32_t kv_free = kv_full + 16;         // [2] the unit's S / dP MMAs are done
+    const uint32_t qdo_full = kv_free + 16;        // [2] Q and dO of a step landed (both copy warps announce bytes)
+    const uint32_t qdo_free = qdo_full + 16;       // [2] the step's dV^T / dK^T MMAs are done
+    const uint32_t sdp_full = qdo_free + 16;       // [2] S and dP of a step computed
+    const uint32_t pds_ready = sdp_full + 16;      // [2] P and dS of a step are in shared memory (8 warps); S / dP have been read
+    const uint32_t pds_free = pds_ready + 16;      // [1] the MMAs that read P and dS are done
+    const uint32_t acc_full = pds_free + 8;        // [2] the unit's sums are complete
+    const uint32_t acc_free = acc_full + 16;       // [2] ... and have been read out of tensor memory
     if (tid == 0) {
         s_abort = (base & 1023u) ? 1 : 0;
         if (s_abort && a.status) atomicOr(a.status, BF1_DEV_WAIT_TIMEOUT);
-        mbar_init(bar_ld, 2);
-        mbar_init(bar_sdp, 1);
-        mbar_init(bar_pds, kRowWarps);
-        mbar_init(bar_acc, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(kv_full + 8 * b, 2);
+            mbar_init(kv_free + 8 * b, 1);
+            mbar_init(qdo_full + 8 * b, 2);
+            mbar_init(qdo_free + 8 * b, 1);
+            mbar_init(sdp_full + 8 * b, 1);
+            mbar_init(pds_ready + 8 * b, 8);
+            mbar_init(acc_full + 8 * b, 1);
+            mbar_init(acc_free + 8 * b, 1);
+        }
+        mbar_init(pds_free, 1);
         fence_mbar_init();
     }
     __syncwarp();
     if (warp == 0) {
-        tmem_alloc(smem_u32(&s_tmem), 256);
+        tmem_alloc(smem_u32(&s_tmem), 512);
         tmem_relinquish();
     }
-    if (a.group == 1) clear_idle_rows<D>(sQ, sDO, tid, kBwdThreads);
+    if (a.group == 1) {   // one head per KV head: rows 64..127 of the Q / dO buffers are never written by a copy
+        clear_idle_rows<D>(base + L::kQ, base + L::kDO, tid, kDkvThreads);
+        clear_idle_rows<D>(base + L::kQ + L::kQBytes, base + L::kDO + L::kQBytes, tid, kDkvThreads);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     volatile int* abort_flag = &s_abort;
-    const int steps = (r_end - r_begin) * pairs;
-    if (s_abort || steps <= 0) {   // (uniform over the CTA)
+    if (s_abort) {   // (uniform over the CTA)
         __syncthreads();
-        if (warp == 0) tmem_dealloc(tmem, 256);
+        if (warp == 0) tmem_dealloc(tmem, 512);
         return;
     }
-    // S and dP are recomputed for every reader; dV^T and dK^T stay where they are until the last one
-    constexpr uint32_t kColS = 0, kColDP = 64, kColDVt = 128, kColDKt = 192;
-    const uint32_t q_tx = a.group > 1 ? L::kQBytes : L::kQBytes / 2;
+    // tensor memory: S | dP of buffer b at columns 128 b; dV^T | dK^T (64 columns each: head dimension on the lanes,
+    // the block's 64 key rows along the columns) of buffer b at 256 + 128 b
+    constexpr uint32_t kColDP = 64, kColAcc = 256, kColDKt = 64;
+    const uint32_t q_tx = a.group > 1 ? L::kQBytes : L::kQBytes / 2;   // one head per KV head: half a tile per copy set
+    const uint32_t sP = base + L::kP, sDS = base + L::kDS;
 
-    if (warp == kWarpLoadA || warp == kWarpLoadB) {
-        // ---- copies: Q and K (first warp), dO and V (second warp) of every step.  P takes over V's buffer and dS
-        // K's at d = 128, so K and V come again for every reader (from L2). ----
-        const bool first = warp == kWarpLoadA;
-        int jq = a.qb_block[a.inv.readers[r_begin]];
-        for (int step = 0; step < steps; ++step) {
-            int jq_next = 0;
-            if (step + 1 < steps) jq_next = a.qb_block[a.inv.readers[r_begin + (step + 1) / pairs]];
-            if (step > 0) mbar_wait(bar_acc, (step - 1) & 1, abort_flag, a.status);
+    if (warp == 0 || warp == 1) {
+        // ---- copies ----
+        const bool first = warp == 0;
+        int s = 0;   // steps so far
+        DkvUnit u = dkv_unit(a, 0, n_units, pairs);
+        for (int n = 0; u.ok; ++n) {
+            const DkvUnit un = dkv_unit(a, n + 1, n_units, pairs);
+            const int b = n & 1;
+            if (n >= 2) mbar_wait(kv_free + 8 * b, ((n >> 1) - 1) & 1, abort_flag, a.status);
             if (elect_one()) {
-                mbar_expect_tx(bar_ld, q_tx + L::kKVBytes);
-                const int head0 = kvh * a.group + (step % pairs) * 2;
-                if (first) {
-                    tma_load_4d(sK, &tm_k, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
-                    load_q_tile<D>(sQ, &tm_q, seq0 + jq * kBlock64, head0, a.group, bar_ld);
-                } else {
-                    tma_load_4d(sV, &tm_v, 0, seq0 + p * kBlock64, kvh, 0, bar_ld);
-                    load_q_tile<D>(sDO, &tm_do, seq0 + jq * kBlock64, head0, a.group, bar_ld);
-                }
+                mbar_expect_tx(kv_full + 8 * b, L::kKVBytes);
+                if (first) tma_load_4d(base + L::kK + b * L::kKVBytes, &tm_k, 0, u.seq0 + u.p * kBlock64, u.kvh, 0, kv_full + 8 * b);
+                else tma_load_4d(base + L::kV + b * L::kKVBytes, &tm_v, 0, u.seq0 + u.p * kBlock64, u.kvh, 0, kv_full + 8 * b);
             }
             __syncwarp();
-            jq = jq_next;
+            int jq = u.steps > 0 ? a.qb_block[a.inv.readers[u.r_begin]] : 0;
+            for (int step = 0; step < u.steps; ++step, ++s) {
+                int jq_next = 0;
+                if (step + 1 < u.steps) jq_next = a.qb_block[a.inv.readers[u.r_begin + (step + 1) / pairs]];
+                const int sb = s & 1;
+                if (s >= 2) mbar_wait(qdo_free + 8 * sb, ((s >> 1) - 1) & 1, abort_flag, a.status);
+                if (elect_one()) {
+                    mbar_expect_tx(qdo_full + 8 * sb, q_tx);
+                    const int head0 = u.kvh * a.group + (step % pairs) * 2;
+                    if (first) load_q_tile<D>(base + L::kQ + sb * L::kQBytes, &tm_q, u.seq0 + jq * kBlock64, head0, a.group, qdo_full + 8 * sb);
+                    else load_q_tile<D>(base + L::kDO + sb * L::kQBytes, &tm_do, u.seq0 + jq * kBlock64, head0, a.group, qdo_full + 8 * sb);
+                }
+                __syncwarp();
+                jq = jq_next;
+            }
+            u = un;
         }
-    } else if (warp == kWarpMma) {
+    } else if (warp == 2 || warp == 3) {
+        // ---- MMAs: warp 2 issues S and dP of every step, warp 3 the two transposed products ----
         constexpr uint32_t kHi = desc_hi_sw128(1024);
         constexpr uint32_t kIdT = idesc_bf16_f32_ab(64, true, true);   // dV^T, dK^T: A and B MN-major
-        for (int step = 0; step < steps; ++step) {
-            mbar_wait(bar_ld, step & 1, abort_flag, a.status);
-            tc_fence_after();
-            if (elect_one()) {
-                issue_s_dp<D>(tmem + kColS, tmem + kColDP, sQ, sDO, sK, sV);
-                mma_commit(bar_sdp);
-            }
-            __syncwarp();
-            mbar_wait(bar_pds, step & 1, abort_flag, a.status);
-            tc_fence_after();
-            if (elect_one()) {
-                // dV^T += dO^T P and dK^T += Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
-                // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
+        int s = 0;
+        DkvUnit u = dkv_unit(a, 0, n_units, pairs);
+        for (int n = 0; u.ok; ++n) {
+            const DkvUnit un = dkv_unit(a, n + 1, n_units, pairs);
+            const int b = n & 1;
+            if (warp == 2) mbar_wait(kv_full + 8 * b, (n >> 1) & 1, abort_flag, a.status);
+            else if (n >= 2) mbar_wait(acc_free + 8 * b, ((n >> 1) - 1) & 1, abort_flag, a.status);
+            for (int step = 0; step < u.steps; ++step, ++s) {
+                const int sb = s & 1;
+                const uint32_t sQ = base + L::kQ + sb * L::kQBytes, sDO = base + L::kDO + sb * L::kQBytes;
+                if (warp == 2) {
+                    mbar_wait(qdo_full + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
+                    // the buffer's last S and dP must have been read
+                    if (s >= 2) mbar_wait(pds_ready + 8 * sb, ((s >> 1) - 1) & 1, abort_flag, a.status);
+                    tc_fence_after();
+                    if (elect_one()) {
+                        issue_s_dp<D>(tmem + sb * 128, tmem + sb * 128 + kColDP, sQ, sDO, base + L::kK + b * L::kKVBytes,
+                                      base + L::kV + b * L::kKVBytes);
+                        mma_commit(sdp_full + 8 * sb);
+                        if (step == u.steps - 1) mma_commit(kv_free + 8 * b);
+                    }
+                    __syncwarp();
+                } else {
+                    mbar_wait(pds_ready + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
+                    tc_fence_after();
+                    if (elect_one()) {
+                        // dV^T += dO^T P and dK^T += Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
+                        // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
+                        const uint32_t t_acc = tmem + kColAcc + b * 128;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t ko = (kk * 2048) >> 4;
-                    if (kk == 0 && step == 0) mma_ss_lohi<false>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                    else mma_ss_lohi<true>(tmem + kColDVt, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                }
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t ko = (kk * 2048) >> 4;
+                            if (kk == 0) {
+                                if (step == 0) mma_ss_lohi<false>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                                else mma_ss_lohi<true>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                            } else {
+                                mma_ss_lohi<true>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                            }
+                        }
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t ko = (kk * 2048) >> 4;
-                    if (kk == 0 && step == 0) mma_ss_lohi<false>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
-                    else mma_ss_lohi<true>(tmem + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t ko = (kk * 2048) >> 4;
+                            if (kk == 0) {
+                                if (step == 0) mma_ss_lohi<false>(t_acc + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                                else mma_ss_lohi<true>(t_acc + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                            } else {
+                                mma_ss_lohi<true>(t_acc + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
+                            }
+                        }
+                        mma_commit(qdo_free + 8 * sb);
+                        mma_commit(pds_free);
+                        if (step == u.steps - 1) mma_commit(acc_full + 8 * b);
+                    }
+                    __syncwarp();
                 }
-                mma_commit(bar_acc);
             }
-            __syncwarp();
+            u = un;
+        }
+    } else if (warp < 12) {
+        // ---- arithmetic on S and dP: two threads per tile row (head hl, token tl of the reader), warps 4-7 on key
+        // columns 0..31 and warps 8-11 on columns 32..63 ----
+        const int half = (warp - 4) >> 2;
+        const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const int row = tid & 127, hl = row >> 6, tl = row & 63;
+        int s = 0;
+        DkvUnit u = dkv_unit(a, 0, n_units, pairs);
+        for (int n = 0; u.ok; ++n) {
+            const DkvUnit un = dkv_unit(a, n + 1, n_units, pairs);
+            // the reader of a step, its block index, the row's LSE (log2 domain) and D_i are fetched one step ahead:
+            // dependent global loads that would otherwise sit between the MMAs and the arithmetic
+            auto fetch = [&](int step, int& g, float& lse2, float& drow) {
+                g = a.inv.readers[u.r_begin + step / pairs];
+                const int jq = a.qb_block[g], pr = step % pairs;
+                const int rows_valid = min(kBlock64, u.seqlen - jq * kBlock64);
+                lse2 = INFINITY;
+                drow = 0.f;
+                if (tl < rows_valid && pr * 2 + hl < a.group) {
+                    const size_t at = (size_t)(u.kvh * a.group + pr * 2 + hl) * a.total_tokens + u.seq0 + jq * kBlock64 + tl;
+                    lse2 = a.lse[at] * 1.4426950408889634f;
+                    drow = a.delta[at];
+                }
+            };
+            int g = 0, g_next = 0;
+            float lse2 = INFINITY, drow = 0.f, lse2_next = INFINITY, drow_next = 0.f;
+            if (u.steps > 0) fetch(0, g, lse2, drow);
+            for (int step = 0; step < u.steps; ++step, ++s) {
+                if (step + 1 < u.steps) fetch(step + 1, g_next, lse2_next, drow_next);
+                const int sb = s & 1;
+                mbar_wait(sdp_full + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
+                tc_fence_after();
+                uint32_t pw[16], dw[16];
+                p_and_ds(t_lane + sb * 128, t_lane + sb * 128 + kColDP, half, tl, g == u.gp, lse2, drow, a.scale, a.scale_log2, pw, dw);
+                if (s >= 1) mbar_wait(pds_free, (s - 1) & 1, abort_flag, a.status);   // the MMAs of the step before have read P and dS
+                store_row_piece(sP + row * 128, row, half, pw);
+                store_row_piece(sDS + row * 128, row, half, dw);
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pds_ready + 8 * sb);
+                g = g_next, lse2 = lse2_next, drow = drow_next;
+            }
+            u = un;
         }
     } else {
-        // ---- row warps: tile row (head hl, token tl of the reader) and which half of the 64 key columns ----
+        // ---- the finished dV^T / dK^T of a unit: lane = head-dimension index, 64 key rows along the columns ----
         const uint32_t t_lane = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        const int row = tid & 127, half = tid >> 7;
-        const int hl = row >> 6, tl = row & 63;
-        // the reader of a step, its block index, the row's LSE (log2 domain) and D_i are fetched one step ahead:
-        // dependent global loads that would otherwise sit between the MMAs and the arithmetic
-        auto fetch = [&](int step, int& g, float& lse2, float& drow) {
-            g = a.inv.readers[r_begin + step / pairs];
-            const int jq = a.qb_block[g], pr = step % pairs;
-            const int rows_valid = min(kBlock64, seqlen - jq * kBlock64);
-            lse2 = INFINITY;
-            drow = 0.f;
-            if (tl < rows_valid && pr * 2 + hl < a.group) {
-                const size_t at = (size_t)(kvh * a.group + pr * 2 + hl) * a.total_tokens + seq0 + jq * kBlock64 + tl;
-                lse2 = a.lse[at] * 1.4426950408889634f;
-                drow = a.delta[at];
-            }
-        };
-        int g, g_next = 0;
-        float lse2, drow, lse2_next = INFINITY, drow_next = 0.f;
-        fetch(0, g, lse2, drow);
-        for (int step = 0; step < steps; ++step) {
-            if (step + 1 < steps) fetch(step + 1, g_next, lse2_next, drow_next);
-            mbar_wait(bar_sdp, step & 1, abort_flag, a.status);
-            tc_fence_after();
-            for (int hh = half * (2 / kPerRow); hh < (half + 1) * (2 / kPerRow); ++hh) {
-                uint32_t pw[16], dw[16];
-                p_and_ds(t_lane + kColS, t_lane + kColDP, hh, tl, g == gp, lse2, drow, a.scale, a.scale_log2, pw, dw);
-                store_row_piece(sP + row * 128, row, hh, pw);
-                store_row_piece(sDS + row * 128, row, hh, dw);
-            }
-            fence_proxy_async();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pds);
-            g = g_next, lse2 = lse2_next, drow = drow_next;
-        }
-        mbar_wait(bar_acc, (steps - 1) & 1, abort_flag, a.status);
-        tc_fence_after();
-
-        // ---- dV^T / dK^T: lane = head-dimension index, 64 key rows along the columns ----
-        if (row < D) {   // d = 64: lanes 64..127 hold nothing (warp-uniform)
-            const size_t rstride = (size_t)a.hkv * D;
-            const size_t row0 = ((size_t)(seq0 + p * kBlock64) * a.hkv + kvh) * D + row;
-            float* pk = part >= 0 ? a.partial + (((size_t)part * a.hkv + kvh) * 2) * (kBlock64 * D) + row : nullptr;
-            for (int hh = half * (2 / kPerRow); hh < (half + 1) * (2 / kPerRow); ++hh) {
-                uint32_t vr[32], kr[32];
-                tmem_ld32(t_lane + kColDVt + hh * 32, vr);
-                tmem_ld32(t_lane + kColDKt + hh * 32, kr);
-                tmem_wait_ld();
+        const int row = tid & 127;
+        DkvUnit u = dkv_unit(a, 0, n_units, pairs);
+        for (int n = 0; u.ok; ++n) {
+            const DkvUnit un = dkv_unit(a, n + 1, n_units, pairs);
+            const int b = n & 1;
+            if (u.steps > 0) {
+                mbar_wait(acc_full + 8 * b, (n >> 1) & 1, abort_flag, a.status);
+                tc_fence_after();
+                if (row < D) {   // d = 64: lanes 64..127 hold nothing (warp-uniform)
+                    const size_t rstride = (size_t)a.hkv * D;
+                    const size_t row0 = ((size_t)(u.seq0 + u.p * kBlock64) * a.hkv + u.kvh) * D + row;
+                    float* pk = u.part >= 0 ? a.partial + (((size_t)u.part * a.hkv + u.kvh) * 2) * (kBlock64 * D) + row : nullptr;
+#pragma unroll 1
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t vr[32], kr[32];
+                        tmem_ld32(t_lane + kColAcc + b * 128 + hh * 32, vr);
+                        tmem_ld32(t_lane + kColAcc + b * 128 + kColDKt + hh * 32, kr);
+                        tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const int kvr = hh * 32 + c;
-                    if (kvr < kv_valid) {
-                        if (part < 0) {
-                            a.dv[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(vr[c]));
-                            a.dk[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(kr[c]));
-                        } else {
-                            pk[kvr * D] = __uint_as_float(kr[c]);
-                            pk[kBlock64 * D + kvr * D] = __uint_as_float(vr[c]);
+                        for (int c = 0; c < 32; ++c) {
+                            const int kvr = hh * 32 + c;
+                            if (kvr < u.kv_valid) {
+                                if (u.part < 0) {
+                                    a.dv[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(vr[c]));
+                                    a.dk[row0 + kvr * rstride] = __float2bfloat16_rn(__uint_as_float(kr[c]));
+                                } else {
+                                    pk[kvr * D] = __uint_as_float(kr[c]);
+                                    pk[kBlock64 * D + kvr * D] = __uint_as_float(vr[c]);
+                                }
+                            }
                         }
                     }
                 }
+                tc_fence_before();
+                named_sync(1, 128);
+                if ((tid & 127) == 0) mbar_arrive(acc_free + 8 * b);
             }
+            u = un;
         }
-        tc_fence_before();
     }
+    tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 256);
+    if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
 // KV blocks whose readers were cut into several runs: add the runs' partial sums in run order.  Few blocks
@@ -995,8 +1091,8 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
         // two CTAs per SM need the whole shared-memory carve-out
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<128>::kTotal));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<64>::kTotal));
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::kTotal_kv));
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::kTotal_kv));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkvSmem<128>::kTotal));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkvSmem<64>::kTotal));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dq_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
         BF1_CUDA_CHECK(cudaFuncSetAttribute(bwd_dkv_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
@@ -1063,14 +1159,14 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     int sms = 0;
     BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const int grid_q = (int)std::min<int64_t>(sms, (int64_t)cap * hkv * (group == 4 ? 2 : 1));   // persistent: one CTA per SM
-    dim3 grid_kv((unsigned)lay.n_units, hkv);
+    const int grid_kv = (int)std::min<int64_t>(sms, (int64_t)lay.n_units * hkv);
     if (d == 128) {
         bwd_dq_kernel<128><<<grid_q, kDqThreads, DqSmem<128>::kTotal, st>>>(tq, tk, tv, tg, to, a);
-        bwd_dkv_kernel<128><<<grid_kv, kBwdThreads, BwdSmem<128>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
+        bwd_dkv_kernel<128><<<grid_kv, kDkvThreads, DkvSmem<128>::kTotal, st>>>(tq, tk, tv, tg, a);
         bwd_combine_kernel<128><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     } else {
         bwd_dq_kernel<64><<<grid_q, kDqThreads, DqSmem<64>::kTotal, st>>>(tq, tk, tv, tg, to, a);
-        bwd_dkv_kernel<64><<<grid_kv, kBwdThreads, BwdSmem<64>::kTotal_kv, st>>>(tq, tk, tv, tg, a);
+        bwd_dkv_kernel<64><<<grid_kv, kDkvThreads, DkvSmem<64>::kTotal, st>>>(tq, tk, tv, tg, a);
         bwd_combine_kernel<64><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
     }
     BF1_CUDA_CHECK(cudaGetLastError());
