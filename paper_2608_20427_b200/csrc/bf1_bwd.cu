@@ -52,7 +52,9 @@ struct InvPlan {
     int32_t* unit_begin;  // [max_units] its readers: readers[begin .. end)
     int32_t* unit_end;
     int32_t* unit_part;   // [max_units] partial-sum slot it writes, or -1: it writes the final bf16 rows
-    int32_t* scalars;     // [4] number of units, total readers, chunk, partial slots
+    int32_t* unit_order;  // [max_units] units, longest first: the order in which the dK/dV kernel deals them out
+    int32_t* multi;       // [cap] the KV slots whose readers were cut into more than one run
+    int32_t* scalars;     // [8] number of units, total readers, chunk, partial slots, slots in `multi`
     int32_t cap, max_units;
 };
 
@@ -88,23 +90,22 @@ __device__ __forceinline__ int list_entry(const int32_t* list, int e, int cnt, i
 
 // ---- pieces shared by the two compute kernels ------------------------------------------------------------------
 
-// S = Q K^T and dP = dO V^T: D / 16 k-steps over the head dimension (one thread).
+// S = Q K^T (or dP = dO V^T): D / 16 k-steps over the head dimension, 128 x 64 output, A and B K-major (one thread).
+template <int D>
+__device__ __forceinline__ void issue_qk(uint32_t t_out, uint32_t sA, uint32_t sB) {
+    constexpr uint32_t kHi = desc_hi_sw128(1024);
+    constexpr uint32_t kIdS = idesc_bf16_f32_ab(64, false, false);
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
+        if (kk == 0) mma_ss_lohi<false>(t_out, desc_lo_sw128(sA, 16) + a_off, desc_lo_sw128(sB, 16) + b_off, kHi, kIdS);
+        else mma_ss_lohi<true>(t_out, desc_lo_sw128(sA, 16) + a_off, desc_lo_sw128(sB, 16) + b_off, kHi, kIdS);
+    }
+}
 template <int D>
 __device__ __forceinline__ void issue_s_dp(uint32_t t_s, uint32_t t_dp, uint32_t sQ, uint32_t sDO, uint32_t sK, uint32_t sV) {
-    constexpr uint32_t kHi = desc_hi_sw128(1024);
-    constexpr uint32_t kIdS = idesc_bf16_f32_ab(64, false, false);     // 128 x 64, A and B K-major
-#pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
-        if (kk == 0) mma_ss_lohi<false>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
-        else mma_ss_lohi<true>(t_s, desc_lo_sw128(sQ, 16) + a_off, desc_lo_sw128(sK, 16) + b_off, kHi, kIdS);
-    }
-#pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t a_off = ((kk / 4) * 16384 + (kk % 4) * 32) >> 4, b_off = ((kk / 4) * 8192 + (kk % 4) * 32) >> 4;
-        if (kk == 0) mma_ss_lohi<false>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
-        else mma_ss_lohi<true>(t_dp, desc_lo_sw128(sDO, 16) + a_off, desc_lo_sw128(sV, 16) + b_off, kHi, kIdS);
-    }
+    issue_qk<D>(t_s, sQ, sK);
+    issue_qk<D>(t_dp, sDO, sV);
 }
 
 // P and dS of this thread's 32 columns (half = 0 / 1: columns 0..31 / 32..63) of its row, from S and dP in tensor
@@ -601,7 +602,7 @@ __global__ void __launch_bounds__(256) inverse_route_kernel(const BwdArgs a) {
 // One CTA: offsets of the reader lists, the run length, and the units of the dK/dV kernel.
 __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a) {
     __shared__ int32_t s_warp[32];
-    __shared__ int32_t s_carry[3];
+    __shared__ int32_t s_carry[5];
     __shared__ int32_t s_chunk;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nqb = min(*a.num_qblocks, a.capacity);
@@ -633,7 +634,7 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
         if (tid == 0) s_carry[which] += chunk_total;
         __syncthreads();
     };
-    if (tid < 3) s_carry[tid] = 0;
+    if (tid < 5) s_carry[tid] = 0;
     __syncthreads();
     // pass 1: where each slot's readers start; the total decides the run length
     for (int b0 = 0; b0 < nqb; b0 += 1024) {
@@ -657,10 +658,12 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
         const int g = b0 + tid;
         const int c = g < nqb ? v.count[g] : 0;
         const int runs = (c + chunk - 1) / chunk;
-        int u0, q0;
+        int u0, q0, m0;
         scan(runs, 1, u0);
         scan(runs > 1 ? runs : 0, 2, q0);
+        scan(runs > 1 ? 1 : 0, 3, m0);
         if (g < nqb) {
+            if (runs > 1) v.multi[m0] = g;
             v.chunks[g] = runs;
             v.part0[g] = runs > 1 ? q0 : -1;
             const int first = v.start[g];
@@ -673,6 +676,23 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
             }
         }
     }
+    // units by descending length (a counting sort; which of two equally long units comes first does not matter: the
+    // order only decides which CTA works on which unit)
+    __shared__ int32_t s_bin[1024];
+    s_bin[tid] = 0;
+    __syncthreads();
+    const int n_units = min(s_carry[1], v.max_units);
+    for (int un = tid; un < n_units; un += 1024) atomicAdd(&s_bin[1023 - min(v.unit_end[un] - v.unit_begin[un], 1023)], 1);
+    __syncthreads();
+    {
+        const int c = s_bin[tid];
+        int excl;
+        scan(c, 4, excl);
+        s_bin[tid] = excl;           // where the units of this length start
+    }
+    __syncthreads();
+    for (int un = tid; un < n_units; un += 1024)
+        v.unit_order[atomicAdd(&s_bin[1023 - min(v.unit_end[un] - v.unit_begin[un], 1023)], 1)] = un;
     if (tid == 0) {
         const bool fits = s_carry[1] <= v.max_units && s_carry[2] <= v.cap;
         if (!fits && a.status) atomicOr(a.status, BF1_DEV_CAPACITY);
@@ -680,6 +700,7 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
         v.scalars[1] = s_carry[0];
         v.scalars[2] = chunk;
         v.scalars[3] = s_carry[2];
+        v.scalars[4] = fits ? s_carry[3] : 0;
     }
 }
 
@@ -729,7 +750,7 @@ __device__ __forceinline__ DkvUnit dkv_unit(const BwdArgs& a, int n, int n_units
     u.part = -1;
     if (u.ok) {
         u.kvh = i / n_units;
-        const int unit = i - u.kvh * n_units;
+        const int unit = a.inv.unit_order[i - u.kvh * n_units];
         u.gp = a.inv.unit_slot[unit];
         u.r_begin = a.inv.unit_begin[unit];
         u.steps = (a.inv.unit_end[unit] - u.r_begin) * pairs;
@@ -762,9 +783,11 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
     const uint32_t bars = base + L::kBar;
     const uint32_t kv_full = bars;                 // [2] K and V of a unit landed (both copy warps announce bytes)
     const uint32_t kv_free = kv_full + 16;         // [2] the unit's S / dP MMAs are done
-    const uint32_t qdo_full = kv_free + 16;        // [2] Q and dO of a step landed (both copy warps announce bytes)
-    const uint32_t qdo_free = qdo_full + 16;       // [2] the step's dV^T / dK^T MMAs are done
-    const uint32_t sdp_full = qdo_free + 16;       // [2] S and dP of a step computed
+    const uint32_t q_full = kv_free + 16;          // [2] Q of a step landed
+    const uint32_t do_full = q_full + 16;          // [2] dO of a step landed
+    const uint32_t q_free = do_full + 16;          // [2] the step's dK^T MMAs are done (they come first: S of the step after
+    const uint32_t do_free = q_free + 16;          //     next can then start while its dO is still travelling); [2] its dV^T MMAs
+    const uint32_t sdp_full = do_free + 16;        // [2] S and dP of a step computed
     const uint32_t pds_ready = sdp_full + 16;      // [2] P and dS of a step are in shared memory (8 warps); S / dP have been read
     const uint32_t pds_free = pds_ready + 16;      // [1] the MMAs that read P and dS are done
     const uint32_t acc_full = pds_free + 8;        // [2] the unit's sums are complete
@@ -775,8 +798,10 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
         for (int b = 0; b < 2; ++b) {
             mbar_init(kv_full + 8 * b, 2);
             mbar_init(kv_free + 8 * b, 1);
-            mbar_init(qdo_full + 8 * b, 2);
-            mbar_init(qdo_free + 8 * b, 1);
+            mbar_init(q_full + 8 * b, 1);
+            mbar_init(do_full + 8 * b, 1);
+            mbar_init(q_free + 8 * b, 1);
+            mbar_init(do_free + 8 * b, 1);
             mbar_init(sdp_full + 8 * b, 1);
             mbar_init(pds_ready + 8 * b, 8);
             mbar_init(acc_full + 8 * b, 1);
@@ -830,12 +855,13 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
                 int jq_next = 0;
                 if (step + 1 < u.steps) jq_next = a.qb_block[a.inv.readers[u.r_begin + (step + 1) / pairs]];
                 const int sb = s & 1;
-                if (s >= 2) mbar_wait(qdo_free + 8 * sb, ((s >> 1) - 1) & 1, abort_flag, a.status);
+                const uint32_t full = (first ? q_full : do_full) + 8 * sb;
+                if (s >= 2) mbar_wait((first ? q_free : do_free) + 8 * sb, ((s >> 1) - 1) & 1, abort_flag, a.status);
                 if (elect_one()) {
-                    mbar_expect_tx(qdo_full + 8 * sb, q_tx);
+                    mbar_expect_tx(full, q_tx);
                     const int head0 = u.kvh * a.group + (step % pairs) * 2;
-                    if (first) load_q_tile<D>(base + L::kQ + sb * L::kQBytes, &tm_q, u.seq0 + jq * kBlock64, head0, a.group, qdo_full + 8 * sb);
-                    else load_q_tile<D>(base + L::kDO + sb * L::kQBytes, &tm_do, u.seq0 + jq * kBlock64, head0, a.group, qdo_full + 8 * sb);
+                    if (first) load_q_tile<D>(base + L::kQ + sb * L::kQBytes, &tm_q, u.seq0 + jq * kBlock64, head0, a.group, full);
+                    else load_q_tile<D>(base + L::kDO + sb * L::kQBytes, &tm_do, u.seq0 + jq * kBlock64, head0, a.group, full);
                 }
                 __syncwarp();
                 jq = jq_next;
@@ -857,13 +883,15 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
                 const int sb = s & 1;
                 const uint32_t sQ = base + L::kQ + sb * L::kQBytes, sDO = base + L::kDO + sb * L::kQBytes;
                 if (warp == 2) {
-                    mbar_wait(qdo_full + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
                     // the buffer's last S and dP must have been read
                     if (s >= 2) mbar_wait(pds_ready + 8 * sb, ((s >> 1) - 1) & 1, abort_flag, a.status);
+                    mbar_wait(q_full + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
                     tc_fence_after();
+                    if (elect_one()) issue_qk<D>(tmem + sb * 128, sQ, base + L::kK + b * L::kKVBytes);
+                    __syncwarp();
+                    mbar_wait(do_full + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
                     if (elect_one()) {
-                        issue_s_dp<D>(tmem + sb * 128, tmem + sb * 128 + kColDP, sQ, sDO, base + L::kK + b * L::kKVBytes,
-                                      base + L::kV + b * L::kKVBytes);
+                        issue_qk<D>(tmem + sb * 128 + kColDP, sDO, base + L::kV + b * L::kKVBytes);
                         mma_commit(sdp_full + 8 * sb);
                         if (step == u.steps - 1) mma_commit(kv_free + 8 * b);
                     }
@@ -872,19 +900,9 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
                     mbar_wait(pds_ready + 8 * sb, (s >> 1) & 1, abort_flag, a.status);
                     tc_fence_after();
                     if (elect_one()) {
-                        // dV^T += dO^T P and dK^T += Q^T dS: A = dO / Q MN-major (M = d: 64 per 128-byte row, next 64 at
+                        // dK^T += Q^T dS, then dV^T += dO^T P: A = Q / dO MN-major (M = d: 64 per 128-byte row, next 64 at
                         // +16 KB; K = q rows, 16 per step = 2048 bytes), B = P / dS MN-major (N = 64 kv per row)
                         const uint32_t t_acc = tmem + kColAcc + b * 128;
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t ko = (kk * 2048) >> 4;
-                            if (kk == 0) {
-                                if (step == 0) mma_ss_lohi<false>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                                else mma_ss_lohi<true>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                            } else {
-                                mma_ss_lohi<true>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
-                            }
-                        }
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t ko = (kk * 2048) >> 4;
@@ -895,7 +913,18 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
                                 mma_ss_lohi<true>(t_acc + kColDKt, desc_lo_sw128(sQ, 16384) + ko, desc_lo_sw128(sDS, 16) + ko, kHi, kIdT);
                             }
                         }
-                        mma_commit(qdo_free + 8 * sb);
+                        mma_commit(q_free + 8 * sb);
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t ko = (kk * 2048) >> 4;
+                            if (kk == 0) {
+                                if (step == 0) mma_ss_lohi<false>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                                else mma_ss_lohi<true>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                            } else {
+                                mma_ss_lohi<true>(t_acc, desc_lo_sw128(sDO, 16384) + ko, desc_lo_sw128(sP, 16) + ko, kHi, kIdT);
+                            }
+                        }
+                        mma_commit(do_free + 8 * sb);
                         mma_commit(pds_free);
                         if (step == u.steps - 1) mma_commit(acc_full + 8 * b);
                     }
@@ -998,29 +1027,26 @@ __global__ void __launch_bounds__(kDkvThreads, 1) bwd_dkv_kernel(const __grid_co
 }
 
 // KV blocks whose readers were cut into several runs: add the runs' partial sums in run order.  Few blocks
-// need it (block 0 of a sequence, with the paper's route), so each is spread over gridDim.z CTAs by key rows.
+// need it (block 0 of a sequence, with the paper's route); the work items are (such a block, KV head, one of
+// its key rows), taken round robin by however many CTAs were launched; a thread adds one element of dK or dV.
 template <int D>
-__global__ void __launch_bounds__(256) bwd_combine_kernel(const BwdArgs a) {
-    const int gp = blockIdx.x, kvh = blockIdx.y;
-    if (gp >= min(*a.num_qblocks, a.capacity) || a.inv.scalars[0] == 0) return;
-    const int runs = a.inv.chunks[gp], q0 = a.inv.part0[gp];
-    if (runs <= 1) return;
-    const int seq = a.qb_seq[gp], p = a.qb_block[gp];
-    const int seq0 = a.cu_seqlens[seq];
-    const int kv_valid = min(kBlock64, a.cu_seqlens[seq + 1] - seq0 - p * kBlock64);
-    const int rows_per_cta = (kBlock64 + gridDim.z - 1) / gridDim.z;
-    const int i_lo = blockIdx.z * rows_per_cta * D, i_hi = min(kv_valid, (int)(blockIdx.z + 1) * rows_per_cta) * D;
-    for (int i = i_lo + threadIdx.x; i < i_hi; i += 256) {
-        float sk = 0.f, sv = 0.f;
-#pragma unroll 4
-        for (int r = 0; r < runs; ++r) {
-            const float* pk = a.partial + (((size_t)(q0 + r) * a.hkv + kvh) * 2) * (kBlock64 * D);
-            sk += pk[i];
-            sv += pk[kBlock64 * D + i];
-        }
-        const size_t o = ((size_t)(seq0 + p * kBlock64 + i / D) * a.hkv + kvh) * D + i % D;
-        a.dk[o] = __float2bfloat16_rn(sk);
-        a.dv[o] = __float2bfloat16_rn(sv);
+__global__ void __launch_bounds__(2 * D) bwd_combine_kernel(const BwdArgs a) {
+    const int items = a.inv.scalars[4] * a.hkv * kBlock64;
+    const int which = threadIdx.x / D, col = threadIdx.x % D;   // 0: dK, 1: dV
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int row = item % kBlock64, kvh = (item / kBlock64) % a.hkv;
+        const int gp = a.inv.multi[item / (kBlock64 * a.hkv)];
+        const int runs = a.inv.chunks[gp], q0 = a.inv.part0[gp];
+        const int seq = a.qb_seq[gp], p = a.qb_block[gp];
+        const int seq0 = a.cu_seqlens[seq];
+        if (row >= a.cu_seqlens[seq + 1] - seq0 - p * kBlock64) continue;   // key row outside the sequence
+        const float* pk = a.partial + (((size_t)q0 * a.hkv + kvh) * 2 + which) * (kBlock64 * D) + row * D + col;
+        const size_t run_stride = (size_t)a.hkv * 2 * kBlock64 * D;
+        float sum = 0.f;
+#pragma unroll 8
+        for (int r = 0; r < runs; ++r) sum += pk[r * run_stride];
+        const size_t o = ((size_t)(seq0 + p * kBlock64 + row) * a.hkv + kvh) * D + col;
+        (which ? a.dv : a.dk)[o] = __float2bfloat16_rn(sum);
     }
 }
 
@@ -1029,7 +1055,7 @@ int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int he
 // Where everything lives in the caller's workspace (256-byte aligned sections).
 struct BwdLayout {
     size_t delta, ints, partial, total;
-    size_t n_count, n_start, n_chunks, n_part0, n_wofs, n_readers, n_units;
+    size_t n_count, n_start, n_chunks, n_part0, n_wofs, n_readers, n_units, n_multi;   // (n_units: also unit_order)
     BwdLayout(int64_t T, int hq, int hkv, int d, int cap, int max_degree) {
         auto up = [](size_t x) { return (x + 255) / 256 * 256; };
         n_count = (size_t)cap;
@@ -1039,9 +1065,10 @@ struct BwdLayout {
         n_wofs = 8 * (size_t)cap;
         n_readers = (size_t)cap * max_degree;
         n_units = 2 * (size_t)cap;
+        n_multi = (size_t)cap;
         delta = 0;
         ints = up((size_t)T * hq * sizeof(float));
-        const size_t n_ints = n_count + n_start + n_chunks + n_part0 + n_wofs + n_readers + 4 * n_units + 4;
+        const size_t n_ints = n_count + n_start + n_chunks + n_part0 + n_wofs + n_readers + 5 * n_units + n_multi + 8;
         partial = ints + up(n_ints * sizeof(int32_t));
         total = partial + up((size_t)cap * hkv * 2 * kBlock64 * d * sizeof(float));
     }
@@ -1146,6 +1173,8 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.inv.unit_begin = ip;       ip += lay.n_units;
     a.inv.unit_end = ip;         ip += lay.n_units;
     a.inv.unit_part = ip;        ip += lay.n_units;
+    a.inv.unit_order = ip;       ip += lay.n_units;
+    a.inv.multi = ip;            ip += lay.n_multi;
     a.inv.scalars = ip;
     a.inv.cap = cap;
     a.inv.max_units = (int32_t)lay.n_units;
@@ -1163,11 +1192,11 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     if (d == 128) {
         bwd_dq_kernel<128><<<grid_q, kDqThreads, DqSmem<128>::kTotal, st>>>(tq, tk, tv, tg, to, a);
         bwd_dkv_kernel<128><<<grid_kv, kDkvThreads, DkvSmem<128>::kTotal, st>>>(tq, tk, tv, tg, a);
-        bwd_combine_kernel<128><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
+        bwd_combine_kernel<128><<<4 * sms, 256, 0, st>>>(a);
     } else {
         bwd_dq_kernel<64><<<grid_q, kDqThreads, DqSmem<64>::kTotal, st>>>(tq, tk, tv, tg, to, a);
         bwd_dkv_kernel<64><<<grid_kv, kDkvThreads, DkvSmem<64>::kTotal, st>>>(tq, tk, tv, tg, a);
-        bwd_combine_kernel<64><<<dim3(cap, hkv, 16), 256, 0, st>>>(a);
+        bwd_combine_kernel<64><<<4 * sms, 128, 0, st>>>(a);
     }
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
