@@ -46,7 +46,7 @@ struct InvPlan {
     int32_t* start;       // [cap + 1] first reader of slot g in `readers`
     int32_t* chunks;      // [cap] runs the slot's readers are cut into
     int32_t* part0;       // [cap] first partial-sum slot of a slot with more than one run, else -1
-    int32_t* wofs;        // [cap * 8] where each of the eight scanning warps writes inside the slot's readers
+    int32_t* wofs;        // [cap * 32] where each of the 32 scanning warps writes inside the slot's readers
     int32_t* readers;     // [cap * max_degree] query slots, ascending per KV slot
     int32_t* unit_slot;   // [max_units] KV slot of the unit
     int32_t* unit_begin;  // [max_units] its readers: readers[begin .. end)
@@ -554,23 +554,24 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
 
 // One CTA per KV slot: its readers are the query slots g >= it of the same sequence whose list names its block
 // (with multiplicity, should a caller's list name a block twice).  The candidates' lists are scanned as one flat
-// array (coalesced), each of the eight warps taking a contiguous eighth of the candidates.  kFill = false counts
+// array (coalesced), each of the 32 warps taking a contiguous part of the candidates.  kFill = false counts
 // (per warp, so that the second pass knows where each warp writes), kFill = true writes the readers in ascending
 // order.
+constexpr int kScanWarps = 32;
 template <bool kFill>
-__global__ void __launch_bounds__(256) inverse_route_kernel(const BwdArgs a) {
-    __shared__ int32_t s_cnt[8];
+__global__ void __launch_bounds__(32 * kScanWarps) inverse_route_kernel(const BwdArgs a) {
+    __shared__ int32_t s_cnt[kScanWarps];
     const int gp = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nqb = min(*a.num_qblocks, a.capacity);
     if (gp >= nqb) return;
     const int seq = a.qb_seq[gp], p = a.qb_block[gp];
     const int nb = (a.cu_seqlens[seq + 1] - a.cu_seqlens[seq] + kBlock64 - 1) / kBlock64;
     const int g_end = min(gp - p + nb, nqb);                 // one past the sequence's last query slot
-    const int span = (g_end - gp + 7) / 8;
+    const int span = (g_end - gp + kScanWarps - 1) / kScanWarps;
     const int g_lo = min(gp + warp * span, g_end), g_hi = min(g_lo + span, g_end);
     const int flat = (g_hi - g_lo) * a.max_degree;           // this warp's part of the flat (slot, entry) array
     int total = 0;
-    int32_t* out = kFill ? a.inv.readers + a.inv.start[gp] + a.inv.wofs[gp * 8 + warp] : nullptr;
+    int32_t* out = kFill ? a.inv.readers + a.inv.start[gp] + a.inv.wofs[gp * kScanWarps + warp] : nullptr;
     for (int f0 = 0; f0 < flat; f0 += 32) {
         const int f = f0 + lane;
         bool match = false;
@@ -590,8 +591,8 @@ __global__ void __launch_bounds__(256) inverse_route_kernel(const BwdArgs a) {
         __syncthreads();
         if (threadIdx.x == 0) {
             int run = 0;
-            for (int w = 0; w < 8; ++w) {
-                a.inv.wofs[gp * 8 + w] = run;
+            for (int w = 0; w < kScanWarps; ++w) {
+                a.inv.wofs[gp * kScanWarps + w] = run;
                 run += s_cnt[w];
             }
             a.inv.count[gp] = run;
@@ -1062,7 +1063,7 @@ struct BwdLayout {
         n_start = (size_t)cap + 1;
         n_chunks = (size_t)cap;
         n_part0 = (size_t)cap;
-        n_wofs = 8 * (size_t)cap;
+        n_wofs = 32 * (size_t)cap;
         n_readers = (size_t)cap * max_degree;
         n_units = 2 * (size_t)cap;
         n_multi = (size_t)cap;
@@ -1180,9 +1181,9 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.inv.max_units = (int32_t)lay.n_units;
     cudaStream_t st = (cudaStream_t)stream;
     // the inverse route (readers of every KV block, cut into units) ...
-    inverse_route_kernel<false><<<cap, 256, 0, st>>>(a);
+    inverse_route_kernel<false><<<cap, 32 * kScanWarps, 0, st>>>(a);
     inverse_units_kernel<<<1, 1024, 0, st>>>(a);
-    inverse_route_kernel<true><<<cap, 256, 0, st>>>(a);
+    inverse_route_kernel<true><<<cap, 32 * kScanWarps, 0, st>>>(a);
     BF1_CUDA_CHECK(cudaGetLastError());
     // ... dQ (and D_i) along the route, dK / dV along its inverse
     int sms = 0;
