@@ -26,9 +26,12 @@
 //                    is cut into runs of `chunk` readers handled by different CTAs; their fp32 partial
 //                    sums are added in run order by bwd_combine_kernel.
 //
-// Both compute kernels are one CTA per unit, two CTAs per SM: four warps work on the tile rows, two issue copies
-// and one issues MMAs; P is rounded to bf16 before the MMAs, as in the forward.  With d = 64 the transposed products still run as
-// M = 128 MMAs: tensor-memory lanes 64..127 then hold nothing of value and are not read.
+// Both compute kernels are persistent: one CTA of 16 warps per SM that takes all of tensor memory (two S/dP
+// buffers and two accumulator buffers) and walks through its share of the units, with warps for copies, for
+// issuing MMAs, for the arithmetic on S and dP and for reading finished sums out, so that copies, MMAs and
+// arithmetic of neighbouring entries and units overlap (see the comment in front of each kernel).  P is rounded
+// to bf16 before the MMAs, as in the forward.  With d = 64 the transposed products still run as M = 128 MMAs:
+// tensor-memory lanes 64..127 then hold nothing of value and are not read.
 #include <cuda.h>
 
 #include <algorithm>
