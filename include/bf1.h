@@ -28,9 +28,9 @@
  *   - GQA: Hq = G * Hkv; query head h reads KV head floor(h / G) (the paper gives only the
  *     head counts, Section 4.1; this is the usual grouped convention).
  *   - Base pointers of Q, K, V, O must be 16-byte aligned.
- *   - Supported geometry: b = 64, d in {64, 128}, G = 2 (Section 4.1's 16 query / 8 KV
- *     heads, Section 3.1's b = 64); the forward entry points also take G = 4.  Anything else
- *     returns BF1_ERR_UNSUPPORTED.
+ *   - Supported geometry, in every entry point: b = 64 (Section 3.1), d in {64, 128},
+ *     G = hq / hkv in {1, 2, 4} (Section 4.1's model has 16 query / 8 KV heads, G = 2).
+ *     Anything else returns BF1_ERR_UNSUPPORTED.
  */
 #ifndef BF1_H_
 #define BF1_H_

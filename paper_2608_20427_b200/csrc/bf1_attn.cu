@@ -3,7 +3,7 @@
 // Work unit = one query block (64 tokens) of one sequence x one KV head.  The G = 2 query
 // heads that share the KV head are stacked into one M = 128 tile (rows 0..63: first head,
 // rows 64..127: second head; with G = 4 the tile is 4 heads x 32 tokens and a query block is two
-// units), because they read the same K/V blocks through the same route
+// units; with G = 1 rows 64..127 are idle), because they read the same K/V blocks through the same route
 // list (the route is per block and the same for all heads, Section 3.1).  For every entry p
 // of the unit's list ("tile"):
 //   S = Q K[p]^T        tcgen05.mma, Q and K[p] in shared memory (TMA, 128-byte swizzle),
