@@ -458,8 +458,8 @@ def decode_sweep(bf1, dev):
 
 
 def run_single_decode(args, bf1, dev):
-    """A few plain decode calls at batch 32, context 32768, each on its own random page table."""
-    hq, hkv, d, batch, n, pool = 16, 8, 128, 32, 32768, 8192
+    """A few plain decode calls at batch `--batch`, context 32768, each on its own random page table."""
+    hq, hkv, d, batch, n, pool = 16, 8, 128, args.batch, 32768, 8192
     g = torch.Generator(device=dev)
     g.manual_seed(778)
     k_pages = torch.randn((pool, 64, hkv, d), generator=g, device=dev, dtype=torch.bfloat16)
@@ -483,7 +483,7 @@ def run_single_decode(args, bf1, dev):
         ts.append(e0.elapsed_time(e1))
     nbytes = int(plans[0].count.sum().item()) * 64 * hkv * d * 2 * 2
     ms = statistics.median(ts[args.warmup:])
-    print(json.dumps({"single": "decode batch 32 context 32768", "ms": ms, "steps": args.steps,
+    print(json.dumps({"single": "decode batch %d context 32768" % batch, "ms": ms, "steps": args.steps,
                       "selected_kv_bytes": nbytes, "gbs_incl_launch_latency": nbytes / ms / 1e6}))
 
 
@@ -739,6 +739,7 @@ def main():
     ap.add_argument("--single", default=None, choices=sorted(I.WORKLOADS),
                     help="only time `--steps` launches of one workload (used for profiling)")
     ap.add_argument("--mode", default="bf1", choices=["bf1", "dense", "decode", "bwd"])
+    ap.add_argument("--batch", type=int, default=32, help="sequences per decode call (with --single ... --mode decode)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.single:
         sys.exit(spawn_ranks(args.gpus))
