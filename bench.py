@@ -331,8 +331,8 @@ def host_route_arrays(lists, n, block=64):
 
 
 def topology_sweep(bf1, dev):
-    """Does the route's topology change the kernel's cost?  (Section 5.1: equal-pair-count BF1, sliding and
-    static-random routes have nearly identical sparse kernel time.)  One 32K layer through routes with about
+    """Does the route's topology change the kernel's cost?  (Section 5.1 reports the same sparse kernel time for BF1 and its
+    sliding and static-random controls of equal pair count.)  One 32K layer through routes with about
     the same number of block pairs: BF1, a sliding window with the closest pair count, a seeded static-random
     non-local graph with exactly BF1's list lengths (uploaded from the host, not planned), BF1 without block
     0, dyadic predecessors without a local window.  Kernel time from a CUDA graph of 16 launches; reported
