@@ -104,6 +104,31 @@ def test_gradients_over_other_routes(route):
         assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
 
 
+def test_gradients_of_many_short_sequences():
+    """Hundreds of sequences of one to three blocks: more units than the persistent kernels have CTAs, nearly all of
+    one or two list entries, so every ring, buffer pair and barrier phase changes hands at every step; units of
+    sequences with a single token have nothing but the self block."""
+    rng = np.random.default_rng(77)
+    lens = [int(x) for x in rng.integers(1, 190, size=700)]
+    lens[5] = 0
+    lens[100:108] = [1, 64, 65, 128, 129, 1, 63, 2]
+    w = I.custom(lens, hq=4, hkv=2, d=64, seed=6600)
+    res = run_case(w, seed=7)
+    print(len(lens), sum(lens), res)
+    for name, (rms, mx) in res.items():
+        assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
+
+
+def test_gradients_over_a_dense_route():
+    """Every predecessor selected (lists of up to 32 entries, every block with many readers): long units in the dQ
+    kernel, every KV block of the first half cut into runs in the dK/dV kernel."""
+    w = I.custom([2048], hq=4, hkv=2, d=128, seed=6700, local_blocks=64, global_first=1, dyadic=1)
+    res = run_case(w, seed=8)
+    print(res)
+    for name, (rms, mx) in res.items():
+        assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
+
+
 def test_backward_is_bitwise_reproducible():
     """No floating-point atomics: two runs give the same bits, whatever the workspace held before (block 0 of the
     long sequence has 64 readers and goes through the partial-sum path)."""
