@@ -10,18 +10,22 @@
 // names plan reuse across the epoch as the open problem; here the plan is a ~4 us kernel and is
 // off the per-token path.
 //
-// The work is memory-bound (every selected K/V byte is read once, 2*G MACs per element), so
-// there are no tensor cores here: one CTA per (sequence, KV head, list entry) streams one K page
-// and one V page through shared memory, computes the two grouped query heads' scores and a
-// partial (max, sum, O) triple; the last CTA of a (sequence, KV head) to finish combines the
-// partials (split-KV, combine by atomic ticket) and writes O and LSE.
+// The work is memory-bound (every selected K/V byte is read once, 2*G MACs per element): one kernel,
+// decode_fused_kernel, in which a CTA serves one KV head and one pair of query heads and walks a page
+// list, or a run of it, with an online softmax over a ring of cp.async page pairs.  With enough lists
+// to fill the GPU a CTA takes a whole list; with fewer, every list is cut into runs (about two CTAs per
+// SM in all, down to one page per CTA), each CTA leaves a partial (max, sum, O) in the workspace and
+// the last CTA of a list to finish (atomic ticket, reset by the kernel) adds the runs up in run order.
+#include <algorithm>
+
 #include "bf1_common.cuh"
 
 namespace bf1 {
 
 constexpr int kPage = 64;             // tokens per page = block width b
 constexpr int kDecThreads = 128;
-constexpr int kDecStages = 3;          // page-pair buffers per CTA in the one-CTA-per-list kernel
+constexpr int kDecStages = 3;          // page-pair buffers per CTA
+constexpr int kDecCtasPerSm = 2;       // CTAs aimed at when a list is cut into runs (measured: 1 -> 11.4, 2 -> 10.8, 3 -> 11.7, 6 -> 14.5 us at batch 8)
 
 struct DecodeArgs {
     const __nv_bfloat16* q;           // [batch, hq, d]
@@ -40,174 +44,8 @@ struct DecodeArgs {
     __nv_bfloat16* o;                 // [batch, hq, d]
     float* lse;                       // [hq, batch]
     int32_t batch;
+    int32_t nsplit;                   // decode_fused_kernel: CTAs a page list is cut over (1: no partial results)
 };
-
-template <int D>
-__global__ void __launch_bounds__(kDecThreads) decode_kernel(const DecodeArgs a) {
-    constexpr int kRowWords = D / 2;                    // 32-bit words per K/V row
-    constexpr int kVecPerRow = D / 8;                   // 16-byte vectors per row
-    constexpr int kVecPerThread = kPage * kVecPerRow / kDecThreads;
-    // K rows are read whole by one thread each (16 bytes at a time), so their 16-byte chunks are
-    // XOR-swizzled with the row index to keep 8 neighbouring rows in different banks
-    __shared__ __align__(16) uint32_t sK[kPage][kRowWords];
-    __shared__ __align__(16) uint32_t sV[kPage][kRowWords];
-    __shared__ __align__(16) float sQ[2][D];
-    __shared__ __align__(16) float sP[2][kPage];
-    __shared__ float sRed[2][2];
-    __shared__ float sW[2][64];                         // combine: weight of every partial
-    __shared__ int sLast;
-
-    const int e = blockIdx.x, kvp = blockIdx.y, s = blockIdx.z;
-    const int kvh = kvp / a.pairs, hbase = kvh * a.group + (kvp % a.pairs) * 2;   // first query head of this CTA's pair
-    const int nheads = min(2, a.group - (kvp % a.pairs) * 2);                      // 1 when G = 1
-    const int tid = threadIdx.x;
-    // the four scalars this CTA needs are independent loads: issue them together
-    const int cnt = a.count[s];
-    const int n = a.seqlens[s];
-    const int planned = a.block[s];
-    int pg = a.page[(size_t)s * a.max_degree + e];
-    if (e >= cnt) return;
-    const int j = (n - 1) / kPage;
-    if (j != planned) {               // the plan belongs to another route epoch
-        if (tid == 0 && e == 0 && kvp == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
-        return;
-    }
-    if (pg < 0 || pg >= a.num_pages) {
-        if (tid == 0) atomicOr(a.status, BF1_DEV_BAD_ROUTE);
-        pg = 0;
-    }
-    const int valid = (e == cnt - 1) ? (n - j * kPage) : kPage;   // self page: tokens up to n-1 only
-
-    // ---- stage q (2 heads), the K page and the V page of this KV head: every load of the thread
-    //      is in flight before the first one is used ---------------------------------------------
-    {
-        const size_t row_stride = (size_t)a.hkv * D;    // elements between consecutive tokens of a page
-        const __nv_bfloat16* kp = a.k_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
-        const __nv_bfloat16* vp = a.v_pages + ((size_t)pg * kPage * a.hkv + kvh) * D;
-        uint4 kreg[kVecPerThread], vreg[kVecPerThread];
-#pragma unroll
-        for (int it = 0; it < kVecPerThread; ++it) {
-            const int i = tid + it * kDecThreads, r = i / kVecPerRow, c = i % kVecPerRow;
-            kreg[it] = *reinterpret_cast<const uint4*>(kp + r * row_stride + c * 8);
-            vreg[it] = *reinterpret_cast<const uint4*>(vp + r * row_stride + c * 8);
-        }
-        for (int i = tid; i < 2 * D; i += kDecThreads)
-            sQ[i / D][i % D] = i / D < nheads ? __bfloat162float(a.q[((size_t)s * a.hq + hbase + i / D) * D + i % D]) : 0.f;
-#pragma unroll
-        for (int it = 0; it < kVecPerThread; ++it) {
-            const int i = tid + it * kDecThreads, r = i / kVecPerRow, c = i % kVecPerRow;
-            *reinterpret_cast<uint4*>(&sK[r][(c ^ (r & 7)) * 4]) = kreg[it];
-            *reinterpret_cast<uint4*>(&sV[r][c * 4]) = vreg[it];
-        }
-    }
-    __syncthreads();
-
-    // ---- scores: thread = (head h, key r) ----------------------------------------------------
-    const int h = tid >> 6, r = tid & 63;
-    float sc0 = 0.f, sc1 = 0.f;
-#pragma unroll
-    for (int c = 0; c < kVecPerRow; ++c) {               // 8 elements per step: one 16-byte K load, two of q
-        const uint4 kw = *reinterpret_cast<const uint4*>(&sK[r][(c ^ (r & 7)) * 4]);
-        const float4 qa = *reinterpret_cast<const float4*>(&sQ[h][c * 8]);
-        const float4 qb = *reinterpret_cast<const float4*>(&sQ[h][c * 8 + 4]);
-        sc0 = fmaf(qa.x, __uint_as_float(kw.x << 16), sc0);                  // low half = even element
-        sc1 = fmaf(qa.y, __uint_as_float(kw.x & 0xffff0000u), sc1);
-        sc0 = fmaf(qa.z, __uint_as_float(kw.y << 16), sc0);
-        sc1 = fmaf(qa.w, __uint_as_float(kw.y & 0xffff0000u), sc1);
-        sc0 = fmaf(qb.x, __uint_as_float(kw.z << 16), sc0);
-        sc1 = fmaf(qb.y, __uint_as_float(kw.z & 0xffff0000u), sc1);
-        sc0 = fmaf(qb.z, __uint_as_float(kw.w << 16), sc0);
-        sc1 = fmaf(qb.w, __uint_as_float(kw.w & 0xffff0000u), sc1);
-    }
-    const float sc = (r < valid) ? (sc0 + sc1) * a.scale_log2 : -INFINITY;   // log2 domain
-    float mx = sc;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = mx;
-    __syncthreads();
-    mx = fmaxf(sRed[h][0], sRed[h][1]);                  // finite: key 0 of every page is valid
-    const float p = exp2f(sc - mx);
-    sP[h][r] = p;
-    float sum = p;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-    __syncthreads();                                     // sRed reads done, sP written
-    if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = sum;
-    __syncthreads();
-    sum = sRed[h][0] + sRed[h][1];
-
-    // ---- partial O: thread = (head h, D / 64 adjacent output columns) ---------------------------
-    constexpr int kColsPerThread = D / 64;               // 2 at d = 128 (one 32-bit word of V), 1 at d = 64
-    const int c0 = r * kColsPerThread;
-    float acc[2] = {0.f, 0.f};
-    if (kColsPerThread == 2) {
-        for (int k4 = 0; k4 < valid; k4 += 4) {          // never touch V rows past the newest token
-            const float4 pk = *reinterpret_cast<const float4*>(&sP[h][k4]);   // masked keys: p = 0
-            const float pv[4] = {pk.x, pk.y, pk.z, pk.w};
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                if (k4 + q4 < valid) {
-                    const uint32_t vw = sV[k4 + q4][r];
-                    acc[0] = fmaf(pv[q4], __uint_as_float(vw << 16), acc[0]);
-                    acc[1] = fmaf(pv[q4], __uint_as_float(vw & 0xffff0000u), acc[1]);
-                }
-            }
-        }
-    } else {
-        const __nv_bfloat16* sVh = reinterpret_cast<const __nv_bfloat16*>(&sV[0][0]);
-#pragma unroll 8
-        for (int k = 0; k < valid; ++k) acc[0] = fmaf(sP[h][k], __bfloat162float(sVh[k * D + c0]), acc[0]);
-    }
-    float* my = a.part + ((((size_t)s * a.hkv * a.pairs + kvp) * a.max_degree + e) * 2 + h) * (D + 2);
-#pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c) my[c0 + c] = acc[c];
-    if (r == 0) { my[D] = mx; my[D + 1] = sum; }
-
-    // ---- the last CTA of this (sequence, KV head) combines --------------------------------------
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int t = atomicAdd(a.ticket + s * a.hkv * a.pairs + kvp, 1);
-        sLast = (t == cnt - 1);
-        if (sLast) a.ticket[s * a.hkv * a.pairs + kvp] = 0;   // ready for the next call
-    }
-    __syncthreads();
-    if (!sLast) return;
-    __threadfence();
-    const float* base = a.part + (((size_t)s * a.hkv * a.pairs + kvp) * a.max_degree * 2 + h) * (D + 2);
-    const size_t estride = 2 * (D + 2);
-    // every partial's (max, sum) is fetched by its own thread, so the loads overlap
-    if (r < cnt) sW[h][r] = base[r * estride + D];
-    __syncthreads();
-    float m_all = -INFINITY;
-    for (int i = 0; i < cnt && i < 64; ++i) m_all = fmaxf(m_all, sW[h][i]);
-    float wgt = 0.f, lpart = 0.f;
-    if (r < cnt) {
-        wgt = exp2f(sW[h][r] - m_all);
-        lpart = wgt * base[r * estride + D + 1];
-    }
-    __syncthreads();
-    if (r < cnt) sW[h][r] = wgt;
-    float l_all = lpart;                                 // sum over the (at most 64) partials of this head
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xffffffffu, l_all, off);
-    if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = l_all;
-    __syncthreads();
-    l_all = sRed[h][0] + sRed[h][1];
-    float out[2] = {0.f, 0.f};
-#pragma unroll 4
-    for (int i = 0; i < cnt; ++i) {                      // ascending list order: fixed and data-independent
-        const float w = sW[h][i];
-#pragma unroll
-        for (int c = 0; c < kColsPerThread; ++c) out[c] = fmaf(w, base[i * estride + c0 + c], out[c]);
-    }
-    if (h >= nheads) return;                             // G = 1: the second head of the pair does not exist
-    const float inv = 1.f / l_all;
-    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + hbase + h) * D;
-#pragma unroll
-    for (int c = 0; c < kColsPerThread; ++c) orow[c0 + c] = __float2bfloat16_rn(out[c] * inv);
-    if (r == 0) a.lse[(size_t)(hbase + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
-}
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -235,15 +73,13 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
                  : "r"(addr));
 }
 
-// Large batches: one CTA per (sequence, KV head) walks the whole page list.  There are enough CTAs to
-// fill the GPU without splitting a list over CTAs, so the partial results, the ticket and the combine
-// of decode_kernel (three more trips to L2 per page) are not needed.  Pages stream in through a
+// One CTA per (sequence, KV head, pair of query heads[, run of the list]).  Pages stream in through a
 // kDecStages-deep cp.async ring with ONE block-wide synchronisation per page; inside a page each of the
 // four warps owns 16 keys and keeps its own online-softmax state (max, sum, O) for both grouped heads,
 // merged once at the end.  The arithmetic uses warp-level mma (m16n8k16: the two heads are rows 0 and 1
 // of the 16-row operand, the rest is zero): the work is memory-bound, but as scalar FMAs it was a chain
 // of 1500 dependent instructions and five synchronisations per page, which is what bounded the kernel.
-template <int D>
+template <int D, bool kSplit>
 __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeArgs a) {
     constexpr int kRowBytes = D * 2;
     constexpr int kVecPerRow = D / 8;                   // 16-byte chunks per row
@@ -254,6 +90,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
     extern __shared__ __align__(128) uint8_t dsmem[];
     __shared__ float sM[4][2], sL[4][2];
     __shared__ float sO[4][2][D];
+    __shared__ float sW[2][64];                         // combine: weight of every partial
+    __shared__ float sRed[2][2];
+    __shared__ int sLast;
 
     const int kvp = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
     const int kvh = kvp / a.pairs, hbase = kvh * a.group + (kvp % a.pairs) * 2;   // first query head of this CTA's pair
@@ -269,6 +108,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
     }
     const int tail = n - j * kPage;   // valid tokens of the self page (the last list entry)
     const int32_t* pages = a.page + (size_t)s * a.max_degree;
+    // the part of the list this CTA walks: all of it, or the z-th run of `per` entries
+    const int per = kSplit ? (cnt + a.nsplit - 1) / a.nsplit : cnt;
+    const int e_lo = kSplit ? (int)blockIdx.z * per : 0, e_hi = min(cnt, e_lo + per);
+    if (e_lo >= cnt) return;          // fewer runs than CTAs for this sequence
     auto issue_page = [&](int e, int stage) {
         int pg = pages[e];
         if (pg < 0 || pg >= a.num_pages) {
@@ -290,8 +133,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         }
     };
 #pragma unroll
-    for (int e = 0; e < kDecStages - 1; ++e) {
-        if (e < cnt) issue_page(e, e);
+    for (int i = 0; i < kDecStages - 1; ++i) {
+        if (e_lo + i < e_hi) issue_page(e_lo + i, i);
         cp_async_commit();                               // possibly empty: keeps the group count uniform
     }
     // A fragments of Q: rows 0 and 1 of the 16-row operand are the two grouped heads, the rest zero
@@ -310,14 +153,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
     for (int dn = 0; dn < D / 8; ++dn) acc[dn][0] = acc[dn][1] = acc[dn][2] = acc[dn][3] = 0.f;
     const int key0 = warp * 16;                          // this warp's 16 keys of every page
 
-    for (int e = 0; e < cnt; ++e) {
+    for (int e = e_lo; e < e_hi; ++e) {
         cp_async_wait<kDecStages - 2>();                 // page e has landed (for this thread's copies)
         __syncthreads();                                 // ... for everybody's; and page e-1 is no longer read
-        if (e + kDecStages - 1 < cnt) issue_page(e + kDecStages - 1, (e + kDecStages - 1) % kDecStages);
+        if (e + kDecStages - 1 < e_hi) issue_page(e + kDecStages - 1, (e - e_lo + kDecStages - 1) % kDecStages);
         cp_async_commit();
         const int valid = (e == cnt - 1) ? tail : kPage;
         if (key0 >= valid) continue;                     // warp-uniform: none of this warp's keys exists
-        const uint32_t kb = smem_u32(dsmem) + (e % kDecStages) * 2 * kPageBytes, vb = kb + kPageBytes;
+        const uint32_t kb = smem_u32(dsmem) + ((e - e_lo) % kDecStages) * 2 * kPageBytes, vb = kb + kPageBytes;
         // ---- scores of 16 keys: two n-tiles of 8 keys, D / 16 k-steps ----------------------------
         float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
@@ -392,18 +235,69 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         wgt[w] = exp2f(sM[w][h] - m_all);                // 0 for a warp that never saw a valid key
         l_all = fmaf(wgt[w], sL[w][h], l_all);
     }
-    if (h >= nheads) return;                             // G = 1: the second head of the pair does not exist
-    const float inv = 1.f / l_all;
     constexpr int kColsPerThread = D / 64;
-    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + hbase + h) * D;
+    float out[kColsPerThread];
 #pragma unroll
     for (int c = 0; c < kColsPerThread; ++c) {
         const int col = r * kColsPerThread + c;
         float o = 0.f;
 #pragma unroll
         for (int w = 0; w < 4; ++w) o = fmaf(wgt[w], sO[w][h][col], o);
-        orow[col] = __float2bfloat16_rn(o * inv);
+        out[c] = o;
     }
+    if (kSplit) {
+        // ---- this run's (max, sum, O) goes to the workspace; the last CTA of the list to finish adds the runs up in
+        //      run order (fixed and data-independent) ------------------------------------------------------------
+        const int runs = (cnt + per - 1) / per;
+        const int c0 = r * kColsPerThread;
+        const size_t list_id = (size_t)s * a.hkv * a.pairs + kvp;
+        float* my = a.part + ((list_id * a.max_degree + blockIdx.z) * 2 + h) * (D + 2);
+#pragma unroll
+        for (int c = 0; c < kColsPerThread; ++c) my[c0 + c] = out[c];
+        if (r == 0) { my[D] = m_all; my[D + 1] = l_all; }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const int t = atomicAdd(a.ticket + list_id, 1);
+            sLast = (t == runs - 1);
+            if (sLast) a.ticket[list_id] = 0;            // ready for the next call
+        }
+        __syncthreads();
+        if (!sLast) return;
+        __threadfence();
+        const float* base = a.part + (list_id * a.max_degree * 2 + h) * (D + 2);
+        const size_t estride = 2 * (D + 2);
+        if (r < runs) sW[h][r] = base[r * estride + D];  // every run's max is fetched by its own thread
+        __syncthreads();
+        m_all = -INFINITY;
+        for (int i = 0; i < runs && i < 64; ++i) m_all = fmaxf(m_all, sW[h][i]);
+        float w_mine = 0.f, lpart = 0.f;
+        if (r < runs) {
+            w_mine = exp2f(sW[h][r] - m_all);
+            lpart = w_mine * base[r * estride + D + 1];
+        }
+        __syncthreads();
+        if (r < runs) sW[h][r] = w_mine;
+        l_all = lpart;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xffffffffu, l_all, off);
+        if ((tid & 31) == 0) sRed[h][(tid >> 5) & 1] = l_all;
+        __syncthreads();
+        l_all = sRed[h][0] + sRed[h][1];
+#pragma unroll
+        for (int c = 0; c < kColsPerThread; ++c) out[c] = 0.f;
+#pragma unroll 4
+        for (int i = 0; i < runs; ++i) {
+            const float w = sW[h][i];
+#pragma unroll
+            for (int c = 0; c < kColsPerThread; ++c) out[c] = fmaf(w, base[i * estride + c0 + c], out[c]);
+        }
+    }
+    if (h >= nheads) return;                             // G = 1: the second head of the pair does not exist
+    const float inv = 1.f / l_all;
+    __nv_bfloat16* orow = a.o + ((size_t)s * a.hq + hbase + h) * D;
+#pragma unroll
+    for (int c = 0; c < kColsPerThread; ++c) orow[r * kColsPerThread + c] = __float2bfloat16_rn(out[c] * inv);
     if (r == 0) a.lse[(size_t)(hbase + h) * a.batch + s] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
@@ -535,21 +429,32 @@ extern "C" int bf1_decode_fwd(const void* q, const void* k_pages, const void* v_
     int dev = 0;
     BF1_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return fail(BF1_ERR_NO_DEVICE, "device ordinal %d out of range", dev);
+    constexpr int kSmem128 = kDecStages * 2 * 64 * 128 * 2, kSmem64 = kDecStages * 2 * 64 * 64 * 2;
     if (!sm_count[dev]) {
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 128 * 2));
-        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecStages * 2 * 64 * 64 * 2));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem128));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem128));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem64));
+        BF1_CUDA_CHECK(cudaFuncSetAttribute(decode_fused_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem64));
         BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     }
-    if ((int64_t)batch * hkv * pairs >= sm_count[dev]) {
+    const int64_t lists = (int64_t)batch * hkv * pairs;
+    if (lists >= sm_count[dev]) {
         // enough (sequence, KV head) pairs to fill the GPU: one CTA walks a whole list
+        a.nsplit = 1;
         dim3 grid(hkv * pairs, batch);
-        if (d == 128) decode_fused_kernel<128><<<grid, kDecThreads, kDecStages * 2 * 64 * 128 * 2, (cudaStream_t)stream>>>(a);
-        else decode_fused_kernel<64><<<grid, kDecThreads, kDecStages * 2 * 64 * 64 * 2, (cudaStream_t)stream>>>(a);
+        if (d == 128) decode_fused_kernel<128, false><<<grid, kDecThreads, kSmem128, (cudaStream_t)stream>>>(a);
+        else decode_fused_kernel<64, false><<<grid, kDecThreads, kSmem64, (cudaStream_t)stream>>>(a);
     } else {
-        // few pairs: split every list over CTAs (one page each) and combine
-        dim3 grid(plan->max_degree, hkv * pairs, batch);
-        if (d == 128) decode_kernel<128><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
-        else decode_kernel<64><<<grid, kDecThreads, 0, (cudaStream_t)stream>>>(a);
+        // few lists: every list is cut into runs of pages, one CTA each (about two CTAs per SM in all, down to one
+        // page per CTA), and the last CTA of a list to finish adds the runs' partial results up
+        const int64_t want = (kDecCtasPerSm * (int64_t)sm_count[dev] + lists - 1) / lists;
+        a.nsplit = (int)std::min<int64_t>(std::min<int64_t>(want, plan->max_degree), 64);
+        // a run of fewer pages than the ring has stages needs that much less shared memory (more CTAs per SM)
+        const int per_max = (plan->max_degree + a.nsplit - 1) / a.nsplit;
+        const int stages = std::min(per_max, kDecStages);
+        dim3 grid(hkv * pairs, batch, a.nsplit);
+        if (d == 128) decode_fused_kernel<128, true><<<grid, kDecThreads, kSmem128 / kDecStages * stages, (cudaStream_t)stream>>>(a);
+        else decode_fused_kernel<64, true><<<grid, kDecThreads, kSmem64 / kDecStages * stages, (cudaStream_t)stream>>>(a);
     }
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;

@@ -193,8 +193,8 @@ def test_decode_plan_flags_a_sequence_longer_than_its_page_table():
 @pytest.mark.parametrize("hq,hkv", [(8, 2), (3, 3)], ids=["G4", "G1"])
 @pytest.mark.parametrize("batch_kind", ["few", "many"])
 def test_decode_with_four_and_with_one_query_head_per_kv_head(hq, hkv, batch_kind):
-    """G = 4 runs two CTAs (pairs of query heads) per KV head, G = 1 half a pair; both the split kernel
-    (few sequences) and the one-CTA-per-list kernel (many) are exercised."""
+    """G = 4 runs two CTAs (pairs of query heads) per KV head, G = 1 half a pair; both forms of the kernel
+    are exercised: lists cut into runs with a combine (few sequences) and one CTA per list (many)."""
     lens = [1, 64, 65, 257, 1000, 0, 4097] if batch_kind == "few" else [1 + (37 * i) % 700 for i in range(90)]
     w = I.custom(lens, hq=hq, hkv=hkv, d=128, seed=7100 + hq + len(lens))
     q, k, v = I.draw_qkv(w)
