@@ -17,7 +17,7 @@
 //                                                          the threads), B = K_p MN-major; accumulates in TMEM
 //                    It also leaves D_i in the workspace for the second kernel.
 //   bwd_dkv_kernel   unit = (KV block p, KV head, a run of the query blocks that read p): the INVERSE
-//                    route, which three small kernels derive from the lists on every call (any lists: the
+//                    route, which a few small kernels derive from the lists on every call (any lists: the
 //                    planner's or the caller's).  Per reader j (and pair of heads), S and dP as above, then
 //                        dV^T += dO^T P  (d x 64 x 128)    A = dO MN-major, B = P MN-major ([q][kv] tile)
 //                        dK^T += Q^T  dS (d x 64 x 128)    A = Q MN-major,  B = dS MN-major
@@ -49,7 +49,6 @@ struct InvPlan {
     int32_t* start;       // [cap + 1] first reader of slot g in `readers`
     int32_t* chunks;      // [cap] runs the slot's readers are cut into
     int32_t* part0;       // [cap] first partial-sum slot of a slot with more than one run, else -1
-    int32_t* wofs;        // [cap * 32] where each of the 32 scanning warps writes inside the slot's readers
     int32_t* readers;     // [cap * max_degree] query slots, ascending per KV slot
     int32_t* unit_slot;   // [max_units] KV slot of the unit
     int32_t* unit_begin;  // [max_units] its readers: readers[begin .. end)
@@ -555,55 +554,83 @@ __global__ void __launch_bounds__(kDqThreads, 1) bwd_dq_kernel(const __grid_cons
 
 // ---- the inverse route -----------------------------------------------------------------------------------------
 
-// One CTA per KV slot: its readers are the query slots g >= it of the same sequence whose list names its block
-// (with multiplicity, should a caller's list name a block twice).  The candidates' lists are scanned as one flat
-// array (coalesced), each of the 32 warps taking a contiguous part of the candidates.  kFill = false counts
-// (per warp, so that the second pass knows where each warp writes), kFill = true writes the readers in ascending
-// order.
-constexpr int kScanWarps = 32;
+// The readers of KV slot gp are the query slots of the same sequence whose list names its block (with multiplicity,
+// should a caller's list name a block twice).  Transposing the lists is a counting sort by KV slot, linear in the
+// number of list entries: count (one thread per entry), scan (inverse_units_kernel), fill in whatever order the
+// atomics give, then sort every slot's readers ascending -- the order in which the dK/dV kernel adds is thereby the
+// same on every run.
+__device__ __forceinline__ bool inverse_entry(const BwdArgs& a, int nqb, int f, int& g, int& kv) {
+    g = f / a.max_degree;
+    if (g >= nqb) return false;
+    const int e = f - g * a.max_degree;
+    const int cnt = min(max(a.kv_count[g], 1), a.max_degree);
+    if (e >= cnt) return false;
+    const int j = a.qb_block[g];
+    kv = g - j + list_entry(a.kv_idx + (size_t)g * a.max_degree, e, cnt, j);   // slots of a sequence are consecutive
+    return true;
+}
+
+// kFill = false: count[kv] += 1 (count is zero on entry).  kFill = true: count[kv] is counted down again and hands out
+// the places behind start[kv].
 template <bool kFill>
-__global__ void __launch_bounds__(32 * kScanWarps) inverse_route_kernel(const BwdArgs a) {
-    __shared__ int32_t s_cnt[kScanWarps];
-    const int gp = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(256) inverse_route_kernel(const BwdArgs a) {
     const int nqb = min(*a.num_qblocks, a.capacity);
-    if (gp >= nqb) return;
-    const int seq = a.qb_seq[gp], p = a.qb_block[gp];
-    const int nb = (a.cu_seqlens[seq + 1] - a.cu_seqlens[seq] + kBlock64 - 1) / kBlock64;
-    const int g_end = min(gp - p + nb, nqb);                 // one past the sequence's last query slot
-    const int span = (g_end - gp + kScanWarps - 1) / kScanWarps;
-    const int g_lo = min(gp + warp * span, g_end), g_hi = min(g_lo + span, g_end);
-    const int flat = (g_hi - g_lo) * a.max_degree;           // this warp's part of the flat (slot, entry) array
-    int total = 0;
-    int32_t* out = kFill ? a.inv.readers + a.inv.start[gp] + a.inv.wofs[gp * kScanWarps + warp] : nullptr;
-    for (int f0 = 0; f0 < flat; f0 += 32) {
-        const int f = f0 + lane;
-        bool match = false;
-        int g = 0;
-        if (f < flat) {
-            g = g_lo + f / a.max_degree;
-            const int e = f % a.max_degree;
-            const int cnt = min(max(a.kv_count[g], 1), a.max_degree);
-            if (e < cnt) match = list_entry(a.kv_idx + (size_t)g * a.max_degree, e, cnt, a.qb_block[g]) == p;
-        }
-        const unsigned hits = __ballot_sync(0xffffffffu, match);
-        if (kFill && match) out[total + __popc(hits & ((1u << lane) - 1))] = g;
-        total += __popc(hits);
-    }
-    if (!kFill) {
-        if (lane == 0) s_cnt[warp] = total;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int run = 0;
-            for (int w = 0; w < kScanWarps; ++w) {
-                a.inv.wofs[gp * kScanWarps + w] = run;
-                run += s_cnt[w];
-            }
-            a.inv.count[gp] = run;
-        }
+    const int total = nqb * a.max_degree;
+    for (int f = blockIdx.x * 256 + threadIdx.x; f < total; f += gridDim.x * 256) {
+        int g, kv;
+        if (!inverse_entry(a, nqb, f, g, kv)) continue;
+        if (!kFill) atomicAdd(a.inv.count + kv, 1);
+        else a.inv.readers[a.inv.start[kv] + atomicSub(a.inv.count + kv, 1) - 1] = g;
     }
 }
 
-// One CTA: offsets of the reader lists, the run length, and the units of the dK/dV kernel.
+// One CTA per KV slot: its readers ascending.  Up to 32 by ranking inside a warp; more by a bitonic network whose
+// comparators all point the same way, so that a length that is no power of two needs no padding (elements past the end
+// count as +infinity and never move); in shared memory when they fit, else in place.
+constexpr int kSortSmem = 4096;
+__global__ void __launch_bounds__(256) inverse_sort_kernel(const BwdArgs a) {
+    __shared__ int32_t s_v[kSortSmem];
+    const int gp = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+    if (gp >= min(*a.num_qblocks, a.capacity) || a.inv.scalars[0] == 0) return;
+    const int s0 = a.inv.start[gp], c = a.inv.start[gp + 1] - s0;
+    int32_t* r = a.inv.readers + s0;
+    if (c <= 1) return;
+    if (c <= 32) {
+        if (tid >= 32) return;
+        const int v = lane < c ? r[lane] : 0x7fffffff;
+        int rank = 0;
+        for (int j = 0; j < c; ++j) {
+            const int vj = __shfl_sync(0xffffffffu, v, j);
+            rank += (vj < v) || (vj == v && j < lane);
+        }
+        if (lane < c) r[rank] = v;
+        return;
+    }
+    int32_t* v = c <= kSortSmem ? s_v : r;
+    if (c <= kSortSmem) {
+        for (int i = tid; i < c; i += 256) s_v[i] = r[i];
+    }
+    __syncthreads();
+    for (int k = 2; (k >> 1) < c; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < c; i += 256) {
+                const int l = (j == (k >> 1)) ? (i ^ (k - 1)) : (i ^ j);   // first step of a merge: mirrored partner
+                if (l > i && l < c) {
+                    const int x = v[i], y = v[l];
+                    if (x > y) { v[i] = y; v[l] = x; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    if (c <= kSortSmem) {
+        for (int i = tid; i < c; i += 256) r[i] = s_v[i];
+    }
+}
+
+// One CTA: offsets of the reader lists, the run length, and the units of the dK/dV kernel.  kAll: the counting and the
+// filling of the readers as well (few list entries: one launch instead of four).
+template <bool kAll>
 __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a) {
     __shared__ int32_t s_warp[32];
     __shared__ int32_t s_carry[5];
@@ -639,11 +666,19 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
         __syncthreads();
     };
     if (tid < 5) s_carry[tid] = 0;
+    if (kAll) {
+        for (int g = tid; g < nqb; g += 1024) v.count[g] = 0;
+        __syncthreads();
+        for (int f = tid; f < nqb * a.max_degree; f += 1024) {
+            int g, kv;
+            if (inverse_entry(a, nqb, f, g, kv)) atomicAdd(v.count + kv, 1);
+        }
+    }
     __syncthreads();
     // pass 1: where each slot's readers start; the total decides the run length
     for (int b0 = 0; b0 < nqb; b0 += 1024) {
         const int g = b0 + tid;
-        const int c = g < nqb ? v.count[g] : 0;
+        const int c = g < nqb ? __ldcg(v.count + g) : 0;   // (written by atomics: read where they were performed)
         int excl;
         scan(c, 0, excl);
         if (g < nqb) v.start[g] = excl;
@@ -660,7 +695,7 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
     // pass 2: runs per slot -> unit numbers and partial-sum slots
     for (int b0 = 0; b0 < nqb; b0 += 1024) {
         const int g = b0 + tid;
-        const int c = g < nqb ? v.count[g] : 0;
+        const int c = g < nqb ? __ldcg(v.count + g) : 0;   // (written by atomics: read where they were performed)
         const int runs = (c + chunk - 1) / chunk;
         int u0, q0, m0;
         scan(runs, 1, u0);
@@ -705,6 +740,13 @@ __global__ void __launch_bounds__(1024, 1) inverse_units_kernel(const BwdArgs a)
         v.scalars[2] = chunk;
         v.scalars[3] = s_carry[2];
         v.scalars[4] = fits ? s_carry[3] : 0;
+    }
+    if (kAll) {
+        __syncthreads();
+        for (int f = tid; f < nqb * a.max_degree; f += 1024) {
+            int g, kv;
+            if (inverse_entry(a, nqb, f, g, kv)) v.readers[v.start[kv] + atomicSub(v.count + kv, 1) - 1] = g;
+        }
     }
 }
 
@@ -1059,20 +1101,19 @@ int make_map_4d(CUtensorMap* m, const void* ptr, int64_t T, int H, int d, int he
 // Where everything lives in the caller's workspace (256-byte aligned sections).
 struct BwdLayout {
     size_t delta, ints, partial, total;
-    size_t n_count, n_start, n_chunks, n_part0, n_wofs, n_readers, n_units, n_multi;   // (n_units: also unit_order)
+    size_t n_count, n_start, n_chunks, n_part0, n_readers, n_units, n_multi;   // (n_units: also unit_order)
     BwdLayout(int64_t T, int hq, int hkv, int d, int cap, int max_degree) {
         auto up = [](size_t x) { return (x + 255) / 256 * 256; };
         n_count = (size_t)cap;
         n_start = (size_t)cap + 1;
         n_chunks = (size_t)cap;
         n_part0 = (size_t)cap;
-        n_wofs = 32 * (size_t)cap;
         n_readers = (size_t)cap * max_degree;
         n_units = 2 * (size_t)cap;
         n_multi = (size_t)cap;
         delta = 0;
         ints = up((size_t)T * hq * sizeof(float));
-        const size_t n_ints = n_count + n_start + n_chunks + n_part0 + n_wofs + n_readers + 5 * n_units + n_multi + 8;
+        const size_t n_ints = n_count + n_start + n_chunks + n_part0 + n_readers + 5 * n_units + n_multi + 8;
         partial = ints + up(n_ints * sizeof(int32_t));
         total = partial + up((size_t)cap * hkv * 2 * kBlock64 * d * sizeof(float));
     }
@@ -1171,7 +1212,6 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.inv.start = ip;            ip += lay.n_start;
     a.inv.chunks = ip;           ip += lay.n_chunks;
     a.inv.part0 = ip;            ip += lay.n_part0;
-    a.inv.wofs = ip;             ip += lay.n_wofs;
     a.inv.readers = ip;          ip += lay.n_readers;
     a.inv.unit_slot = ip;        ip += lay.n_units;
     a.inv.unit_begin = ip;       ip += lay.n_units;
@@ -1183,14 +1223,21 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.inv.cap = cap;
     a.inv.max_units = (int32_t)lay.n_units;
     cudaStream_t st = (cudaStream_t)stream;
-    // the inverse route (readers of every KV block, cut into units) ...
-    inverse_route_kernel<false><<<cap, 32 * kScanWarps, 0, st>>>(a);
-    inverse_units_kernel<<<1, 1024, 0, st>>>(a);
-    inverse_route_kernel<true><<<cap, 32 * kScanWarps, 0, st>>>(a);
-    BF1_CUDA_CHECK(cudaGetLastError());
-    // ... dQ (and D_i) along the route, dK / dV along its inverse
     int sms = 0;
     BF1_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // the inverse route (readers of every KV block, cut into units) ...
+    if ((int64_t)cap * route->max_degree <= 4096) {
+        inverse_units_kernel<true><<<1, 1024, 0, st>>>(a);   // few entries: count, scan and fill in one CTA
+    } else {
+        BF1_CUDA_CHECK(cudaMemsetAsync(a.inv.count, 0, lay.n_count * sizeof(int32_t), st));
+        const int grid_inv = (int)std::min<int64_t>(((int64_t)cap * route->max_degree + 255) / 256, 4 * (int64_t)sms);
+        inverse_route_kernel<false><<<grid_inv, 256, 0, st>>>(a);
+        inverse_units_kernel<false><<<1, 1024, 0, st>>>(a);
+        inverse_route_kernel<true><<<grid_inv, 256, 0, st>>>(a);
+    }
+    inverse_sort_kernel<<<cap, 256, 0, st>>>(a);
+    BF1_CUDA_CHECK(cudaGetLastError());
+    // ... dQ (and D_i) along the route, dK / dV along its inverse
     const int grid_q = (int)std::min<int64_t>(sms, (int64_t)cap * hkv * (group == 4 ? 2 : 1));   // persistent: one CTA per SM
     const int grid_kv = (int)std::min<int64_t>(sms, (int64_t)lay.n_units * hkv);
     if (d == 128) {
