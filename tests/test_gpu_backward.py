@@ -129,6 +129,54 @@ def test_gradients_over_a_dense_route():
         assert rms <= REL_RMS and mx <= REL_MAX, (name, rms, mx)
 
 
+def test_backward_over_a_damaged_route_is_the_backward_of_the_repaired_route():
+    """Entries outside [0, j], a list that does not end in its query block, counts past the pitch: every kernel of the
+    library reads a list the same repaired way (the forward flags it), so the gradients over the damaged route are,
+    bit for bit, those over the route with the repairs written in -- and nothing faults."""
+    dev = torch.device("cuda:0")
+    w = I.custom([1500, 300], hq=4, hkv=2, d=128, seed=6800)
+    q, k, v = (t.to(dev) for t in I.draw_qkv(w))
+    d_o = torch.randn(q.shape, generator=torch.Generator().manual_seed(9)).to(torch.bfloat16).to(dev)
+    cu = bf1.cu_seqlens_tensor(w.seqlens, dev)
+
+    def grads(damage):
+        route = bf1.plan_route(cu, w.max_seqlen)
+        deg = route.max_degree
+        cnt = route.kv_count.cpu()
+        blk = route.qb_block.cpu()
+        idx = route.kv_idx.cpu().clone()
+        kc = cnt.clone()
+        g1, g2, g3 = 7, 12, 20            # slots of the first sequence (24 blocks)
+        if damage:
+            idx[g1, 0] = 1000             # out of range            -> read as block 0
+            idx[g2, 1] = -5               # negative                -> read as block 0
+            idx[g3, int(cnt[g3]) - 1] = 3 # last entry not the self block -> read as the self block
+            kc[g2] = deg + 50             # count past the pitch    -> cut to the pitch
+        else:
+            idx[g1, 0] = 0
+            idx[g2, 1] = 0
+            idx[g3, int(cnt[g3]) - 1] = int(blk[g3])
+            # kc[g2] cut to the pitch: the entries past the old count are the -1 padding, read as block 0, and the
+            # last one as the self block
+            kc[g2] = deg
+            idx[g2, int(cnt[g2]) - 1] = 0
+            idx[g2, int(cnt[g2]):deg - 1] = 0
+            idx[g2, deg - 1] = int(blk[g2])
+        route.kv_idx.copy_(idx.to(dev))
+        route.kv_count.copy_(kc.to(dev))
+        o, lse = bf1.attn_fwd(q, k, v, cu, w.max_seqlen, route)
+        out = bf1.attn_bwd(q, k, v, o, lse, d_o, cu, w.max_seqlen, route)
+        torch.cuda.synchronize()
+        return out, int(route.status.item())
+
+    bad, status_bad = grads(True)
+    good, status_good = grads(False)
+    assert status_bad & 8 and not status_good & 8
+    for x, y in zip(bad, good):
+        assert torch.isfinite(x.float()).all()
+        assert torch.equal(x, y)
+
+
 def test_backward_is_bitwise_reproducible():
     """No floating-point atomics: two runs give the same bits, whatever the workspace held before (block 0 of the
     long sequence has 64 readers and goes through the partial-sum path)."""
