@@ -64,13 +64,21 @@ enum {
  * predecessors.  `dyadic` adds j - 2^k for every k >= 0 with j - 2^k >= 0; with
  * local_blocks = 2 this is Eq. 1's "r >= 2" set, because 2^0 and 2^1 are the local blocks. */
 typedef struct {
-    int32_t block;         /* b; must be 64                                              */
+    int32_t block;         /* b: 64 (the paper's) or 128, see below                      */
     int32_t local_blocks;  /* W >= 0                                                     */
     int32_t global_first;  /* 0 or 1                                                     */
     int32_t dyadic;        /* 0 or 1                                                     */
 } bf1_route_cfg;
 
-/* A planned route: for every query block of every sequence, the ascending list of KV
+/* Block width.  Every array of a route is kept per TILE of 64 tokens, whatever b is, and the
+ * kernels only ever see tiles.  With b = 64 a tile is a block.  With b = 128, tile t of a sequence
+ * belongs to block j = t / 2; its list holds both tiles of every earlier block of P(j) and the
+ * tiles of block j up to t itself, which selects, token for token, what Eq. 1 selects at b = 128
+ * (earlier blocks in full, the causal triangle inside the self block).  "Query block", "block
+ * index" and "list" below therefore mean tiles and tile indices; bf1_route_capacity returns the
+ * tile count and twice the block-level list length.  The sequence-sharded prefill takes b = 64 only.
+ *
+ * A planned route: for every query block of every sequence, the ascending list of KV
  * block indices it reads (sequence-local; the last entry is the query block itself), the
  * list length, and the number of selected token pairs (Proposition 1's accounting: a
  * non-self block gives rows*b pairs, the self block rows*(rows+1)/2, rows = tokens in the
@@ -178,7 +186,9 @@ int bf1_attn_fwd_noalloc(const void *q, const void *k, const void *v, const int3
  * paged: k_pages / v_pages are [num_pages, 64, hkv, d] bf16 and page_table[s, i] names the
  * physical page that holds logical block i of sequence s.  The page list changes only when n
  * crosses a block boundary, so one plan serves a whole 64-token route epoch (Section 5.4 names
- * keeping a plan alive across such an epoch as the open systems problem). */
+ * keeping a plan alive across such an epoch as the open systems problem).  Pages stay 64 tokens
+ * with b = 128: a listed block is then two pages, the newest token's own block its pages up to the
+ * one that holds the token, and a plan still serves 64 tokens. */
 typedef struct {
     int32_t  max_degree;   /* host: row pitch of `page`                                          */
     int32_t *count;        /* [batch] pages to read for the sequence (0 for an empty sequence)   */

@@ -314,8 +314,12 @@ __global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_t
         int32_t* list = plan.page + (size_t)s * plan.max_degree;
         int deg = 0;
         int bad = 0;
-        const int j = n > 0 ? (n - 1) / kPage : -1;
-        if (n < 0 || j >= max_pages_per_seq) bad = BF1_DEV_BAD_SEQLENS;
+        // Pages are 64 tokens whatever the route block width b: with b = 128 a listed block is two pages, and
+        // the newest token's own block is its pages up to the one that holds the token.
+        const int f = cfg.block / kPage;
+        const int jt = n > 0 ? (n - 1) / kPage : -1;      // logical page of the newest token
+        const int j = jt >= 0 ? jt / f : -1;              // its route block
+        if (n < 0 || jt >= max_pages_per_seq) bad = BF1_DEV_BAD_SEQLENS;
         if (n > 0 && !bad) {
             int last = -1, kmax = -1;
             if (cfg.dyadic) while ((1 << (kmax + 1)) <= j) ++kmax;
@@ -331,9 +335,12 @@ __global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_t
                 if (m == dcur) --k;
                 if (m == lcur) ++l;
                 if (m != last) {
-                    if (deg < plan.max_degree) list[deg] = page_table[(size_t)s * max_pages_per_seq + m];
-                    else bad |= BF1_DEV_CAPACITY;
-                    ++deg;
+                    const int t1 = (m < j) ? m * f + f - 1 : jt;
+                    for (int t = m * f; t <= t1; ++t) {
+                        if (deg < plan.max_degree) list[deg] = page_table[(size_t)s * max_pages_per_seq + t];
+                        else bad |= BF1_DEV_CAPACITY;
+                        ++deg;
+                    }
                     last = m;
                 }
             }
@@ -341,7 +348,7 @@ __global__ void plan_decode_kernel(const int32_t* seqlens, const int32_t* page_t
         }
         for (int e2 = deg; e2 < plan.max_degree; ++e2) list[e2] = -1;
         plan.count[s] = bad ? 0 : deg;
-        plan.block[s] = j;
+        plan.block[s] = jt;
         if (bad) atomicOr(&s_bad, bad);
     }
     __syncthreads();

@@ -169,6 +169,7 @@ __global__ void __launch_bounds__(kShardThreads, 1) plan_shard_kernel(const Shar
 
 static int check_shard(int64_t n_tokens, const bf1_route_cfg* cfg, int32_t lo_block, int32_t hi_block) {
     if (int rc = check_cfg(cfg)) return rc;
+    if (cfg->block != 64) return fail(BF1_ERR_UNSUPPORTED, "sequence sharding is built for b = 64 only (block width %d)", cfg->block);
     if (n_tokens < 1 || n_tokens > 0x7fffffffLL - 64) return fail(BF1_ERR_INVALID_ARG, "n_tokens %lld out of range", (long long)n_tokens);
     const int64_t nb = (n_tokens + cfg->block - 1) / cfg->block;
     if (lo_block < 0 || hi_block <= lo_block || hi_block > nb)

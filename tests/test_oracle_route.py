@@ -161,6 +161,23 @@ def test_token_mask_structure():
                 assert not tile.any()
 
 
+@pytest.mark.parametrize("b", [64, 128])
+def test_token_mask_at_both_block_widths_equals_eq1_token_by_token(b):
+    """The block width is a parameter of the method: token i (block i // b) sees token c (block c // b)
+    iff c <= i and c's block is in P(i's block), Eq. 1 written out per token pair."""
+    n = 5 * 128 + 70   # a partial last block at either width
+    got = O.token_mask(O.cfg(block=b), n)
+    want = np.zeros((n, n), dtype=bool)
+    for i in range(n):
+        sel = set(generator_P(i // b))
+        for c in range(i + 1):
+            want[i, c] = (c // b) in sel
+    assert (got == want).all()
+    _, cnt, pairs, total = O.route(O.cfg(block=b), n)
+    assert total == int(want.sum()) == int(pairs.sum())
+    assert [int(x) for x in cnt] == [len(generator_P(j)) for j in range((n + b - 1) // b)]
+
+
 def test_closed_form_totals_all_lengths():
     c = O.cfg()
     for n in list(range(1, 4097, 7)) + [64, 128, 192, 193, 256, 257, 1000, 4096]:
