@@ -26,8 +26,9 @@
 //               and queues it for the producer -- all of it global-memory latency that must not
 //               sit in front of the copies,
 //   warps 4-7   softmax, one thread per tile row,
-//   warps 8-11  epilogue: take the finished O out of tensor memory, normalise, store O and LSE,
-//               while the softmax warps are already on the next unit.
+//   warps 8-11  epilogue: take the finished O out of tensor memory into registers (which frees O for the
+//               next unit's first PV), normalise, store O and LSE, while the softmax warps are already
+//               on the next unit.
 // All hand-offs are mbarriers; every wait is bounded (see mbar_wait).
 #include <cuda.h>
 
@@ -42,7 +43,7 @@ constexpr int kThreads = 384;         // 12 warps
 // unit a CTA holds in advance is a unit another CTA cannot take at the end of the launch: with three
 // the last CTAs finished 20 us after the first at 32K, and 8K was 7 % slower.
 constexpr int kQueue = 1;
-constexpr int kRegsCtl = 40, kRegsSoftmax = 144, kRegsEpilogue = 56;   // registers per thread of each warpgroup
+constexpr int kRegsCtl = 40, kRegsSoftmax = 120, kRegsEpilogue = 80;   // registers per thread of each warpgroup
 static_assert(kRegsCtl + kRegsSoftmax + kRegsEpilogue <= 240, "register budgets must fit the launch allocation");
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row
                                             // maximum grows by more than 2^8
@@ -570,13 +571,13 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                         mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
                         tc_fence_after();
 #pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t oreg[32];
-                            tmem_ld32(t_lane + C::kColO + c * 32, oreg);
+                        for (int c = 0; c < D / 16; ++c) {
+                            uint32_t oreg[16];
+                            tmem_ld16(t_lane + C::kColO + c * 16, oreg);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
-                            tmem_st32(t_lane + C::kColO + c * 32, oreg);
+                            for (int e = 0; e < 16; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
+                            tmem_st16(t_lane + C::kColO + c * 16, oreg);
                         }
                     }
                 }
@@ -644,56 +645,53 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             const bool head_ok = hl < args.group;      // G = 1: tile rows 64..127 belong to no head (warp-uniform)
             const bool store = tl < rows_valid && head_ok;
             __nv_bfloat16* orow = args.o + ((size_t)tok * args.hq + (kvh * args.group + hl)) * D;
-            // Full blocks leave through shared memory and TMA stores: each warp packs 32 rows x 32
-            // columns into its own 2 KB staging tile (64-byte swizzle, conflict-free) and one lane
-            // hands it to the copy engine.  Scattered 16-byte global stores from here would sit in the
-            // same load/store path as every other warp's mbarrier and shared-memory traffic and
-            // slow the whole SM down.  16 columns at a time keeps the register budget small.
-            const bool full_tile = rows_valid == (1 << args.r_shift) && head_ok;   // warp-uniform
-            const uint32_t stage_w = base + C::kStageOff + (warp & 3) * 2048;
-            const uint32_t srow = stage_w + lane * 64;
+            // O leaves tensor memory first, all of it, normalised and packed to bf16 in registers: the
+            // next unit's first PV overwrites O and waits for exactly this, so nothing slow (staging,
+            // copy-engine waits) may sit in front of the release.
+            uint32_t pk[D / 2];
 #pragma unroll
             for (int c = 0; c < D / 16; ++c) {
-                if (full_tile && (c & 1) == 0) {
-                    if (lane == 0) bulk_wait_read0();   // the previous store has finished reading the tile
-                    __syncwarp();
-                }
                 uint32_t oreg[16];
                 tmem_ld16(t_lane + C::kColO + c * 16, oreg);
                 tmem_wait_ld();
-                if (c == D / 16 - 1) {   // O has been read out: the next unit may overwrite it
-                    tc_fence_before();
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    pk[c * 8 + e] = pack_bf16x2(__uint_as_float(oreg[2 * e]) * inv_l, __uint_as_float(oreg[2 * e + 1]) * inv_l);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_o_free);
+            // Full blocks then go through shared memory and TMA stores: each warp packs 32 rows x 32
+            // columns into its own 2 KB staging tile (64-byte swizzle, conflict-free) and one lane
+            // hands it to the copy engine.  Scattered 16-byte global stores from here would sit in the
+            // same load/store path as every other warp's mbarrier and shared-memory traffic and
+            // slow the whole SM down.
+            const bool full_tile = rows_valid == (1 << args.r_shift) && head_ok;   // warp-uniform
+            const uint32_t stage_w = base + C::kStageOff + (warp & 3) * 2048;
+            const uint32_t srow = stage_w + lane * 64;
+            if (full_tile) {
+                const int sw = (lane >> 1) & 3;       // 64-byte swizzle: chunk ^= (row / 2) % 4
+#pragma unroll
+                for (int c2 = 0; c2 < D / 32; ++c2) {   // 32 columns = 16 packed registers per store
+                    if (lane == 0) bulk_wait_read0();   // the previous store has finished reading the tile
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_o_free);
-                }
-                uint4 w0, w1;
-                w0.x = pack_bf16x2(__uint_as_float(oreg[0]) * inv_l, __uint_as_float(oreg[1]) * inv_l);
-                w0.y = pack_bf16x2(__uint_as_float(oreg[2]) * inv_l, __uint_as_float(oreg[3]) * inv_l);
-                w0.z = pack_bf16x2(__uint_as_float(oreg[4]) * inv_l, __uint_as_float(oreg[5]) * inv_l);
-                w0.w = pack_bf16x2(__uint_as_float(oreg[6]) * inv_l, __uint_as_float(oreg[7]) * inv_l);
-                w1.x = pack_bf16x2(__uint_as_float(oreg[8]) * inv_l, __uint_as_float(oreg[9]) * inv_l);
-                w1.y = pack_bf16x2(__uint_as_float(oreg[10]) * inv_l, __uint_as_float(oreg[11]) * inv_l);
-                w1.z = pack_bf16x2(__uint_as_float(oreg[12]) * inv_l, __uint_as_float(oreg[13]) * inv_l);
-                w1.w = pack_bf16x2(__uint_as_float(oreg[14]) * inv_l, __uint_as_float(oreg[15]) * inv_l);
-                if (full_tile) {
-                    const int ch = (c & 1) * 2;           // 16-byte chunk inside the 64-byte staging row
-                    const int sw = (lane >> 1) & 3;       // 64-byte swizzle: chunk ^= (row / 2) % 4
-                    st_shared_v4(srow + (((ch + 0) ^ sw) << 4), w0.x, w0.y, w0.z, w0.w);
-                    st_shared_v4(srow + (((ch + 1) ^ sw) << 4), w1.x, w1.y, w1.z, w1.w);
-                    if (c & 1) {
-                        fence_proxy_async();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_3d(&tm_o, (c >> 1) * 32, kvh * args.group + hl, tok0 + ((quarter * 32) & ((1 << args.r_shift) - 1)),
-                                         stage_w);
-                            bulk_commit_group();
-                        }
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch)
+                        st_shared_v4(srow + ((ch ^ sw) << 4), pk[c2 * 16 + ch * 4 + 0], pk[c2 * 16 + ch * 4 + 1],
+                                     pk[c2 * 16 + ch * 4 + 2], pk[c2 * 16 + ch * 4 + 3]);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&tm_o, c2 * 32, kvh * args.group + hl, tok0 + ((quarter * 32) & ((1 << args.r_shift) - 1)),
+                                     stage_w);
+                        bulk_commit_group();
                     }
-                } else if (store) {
-                    // partial last block of a sequence: the rows after it belong to someone else
-                    *reinterpret_cast<uint4*>(orow + c * 16) = w0;
-                    *reinterpret_cast<uint4*>(orow + c * 16 + 8) = w1;
                 }
+            } else if (store) {
+                // partial last block of a sequence: the rows after it belong to someone else
+#pragma unroll
+                for (int c = 0; c < D / 8; ++c)
+                    *reinterpret_cast<uint4*>(orow + c * 8) = make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
             }
             if (store) {
                 const float lse2 = m_used * c2 + lg2_approx(l_run);   // log2 domain
