@@ -187,11 +187,6 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
             }
         }
     };
-    if (args.status && (*args.status & BF1_DEV_WAIT_TIMEOUT)) {   // an earlier launch gave up
-        retire();
-        return;
-    }
-
     const uint32_t base = smem_u32(smem);
     const uint32_t sQ = base + C::kQOff;
     const uint32_t sRing = base + C::kRingOff;
@@ -217,15 +212,20 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
     int* s_nqb = reinterpret_cast<int*>(smem + C::kMiscOff + 8);
 
     if (tid == 0) {
-        *s_abort = 0;
+        // The status word and the block count are read together (two independent loads in flight), and no other
+        // warp waits for them before its own set-up.  If an earlier launch on this status word gave up, this one
+        // raises its abort flag: every role then sees an empty queue and the CTA leaves through the normal exit.
+        const int earlier = args.status ? *args.status : 0;
+        int nqb = 0;
+        if (!args.dense) {
+            nqb = min(*args.num_qblocks, args.capacity);
+        }
+        *s_abort = (earlier & BF1_DEV_WAIT_TIMEOUT) ? 1 : 0;
         if (base & 1023u) {   // the swizzled tiles need a 1024-byte aligned window
             *s_abort = 1;
             if (args.status) atomicOr(args.status, BF1_DEV_WAIT_TIMEOUT);
         }
-        int nqb = 0;
-        if (!args.dense) {
-            nqb = min(*args.num_qblocks, args.capacity);
-        } else {
+        if (args.dense) {
             for (int s = 0; s < args.batch; ++s)
                 nqb += (args.cu_seqlens[s + 1] - args.cu_seqlens[s] + kBlock - 1) / kBlock;
         }
