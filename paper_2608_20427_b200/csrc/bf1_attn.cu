@@ -9,7 +9,7 @@
 //   S = Q K[p]^T        tcgen05.mma, Q and K[p] in shared memory (TMA, 128-byte swizzle),
 //                       fp32 accumulator in tensor memory (two S buffers, ping-pong),
 //   online softmax      one thread per row: tcgen05.ld S, causal mask on the self block only,
-//                       running max / sum in the exp2 domain, P -> bf16 -> tcgen05.st over S,
+//                       reference maximum (moved lazily) / sum in the exp2 domain, P -> bf16 -> tcgen05.st over S,
 //   O += P V[p]         tcgen05.mma with P read from tensor memory and V from shared memory,
 // then O / l is written as bf16 and LSE = max + ln(sum) as fp32.
 // With `dense = 1` the list is replaced by 0..j: plain causal attention through the same code.
@@ -45,8 +45,8 @@ constexpr int kThreads = 384;         // 12 warps
 constexpr int kQueue = 1;
 constexpr int kRegsCtl = 40, kRegsSoftmax = 120, kRegsEpilogue = 80;   // registers per thread of each warpgroup
 static_assert(kRegsCtl + kRegsSoftmax + kRegsEpilogue <= 240, "register budgets must fit the launch allocation");
-constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when the row
-                                            // maximum grows by more than 2^8
+constexpr float kSumGuard = 1.152921504606846976e18f;   // 2^60: a tile whose row sum reaches this (or is not finite)
+                                                        // is redone against its own maximum
 
 struct AttnArgs {
     const int32_t* cu_seqlens;
@@ -535,68 +535,81 @@ __global__ void __launch_bounds__(kThreads, 2) attn_fwd_kernel(const __grid_cons
                 const uint32_t t_s = t_lane + C::kColS + (g & 1) * 64;
                 mbar_wait(bar_s_full + 8 * (g & 1), (g >> 1) & 1, abort_flag, args.status);
                 tc_fence_after();
-                uint32_t sreg[64];
-                {
-                    uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sreg[0]);
-                    uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sreg[32]);
-                    tmem_ld32(t_s, lo);
-                    tmem_ld32(t_s + 32, hi);
-                }
-                tmem_wait_ld();
-                if (i == cnt - 1) {   // self block: causal triangle (warp-uniform branch)
+                // The exponentials of a tile are taken against the row's current reference maximum m_used; the
+                // tile's own maximum is only computed for the first tile of a unit, and again (second pass) when
+                // a row's sum shows that the reference has fallen too far behind (sum >= 2^60, or not finite).
+                // Any reference gives the same softmax as long as nothing overflows: P (bf16), l and O (fp32) are
+                // floating point, so their relative accuracy does not depend on the scale.  The second pass is
+                // entered by the whole warp (its tensor-memory accesses are warp-wide), but only a row whose own
+                // sum tripped moves its reference; every other row multiplies by exactly 1 and recomputes the
+                // values it already had, so a row's arithmetic depends on that row alone (later tokens of the
+                // block cannot change it).
+                uint32_t preg[32];
+                float tile_sum = 0.f;
+                bool tripped = false;
+#pragma unroll 1
+                for (int pass = 0; pass < 2; ++pass) {
+                    uint32_t sreg[64];
+                    {
+                        uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sreg[0]);
+                        uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sreg[32]);
+                        tmem_ld32(t_s, lo);
+                        tmem_ld32(t_s + 32, hi);
+                    }
+                    tmem_wait_ld();
+                    if (i == cnt - 1) {   // self block: causal triangle (warp-uniform branch)
 #pragma unroll
-                    for (int c = 0; c < 64; ++c)
-                        if (c > tl) sreg[c] = 0xff800000u;   // -inf
-                }
-                float mxa = -INFINITY, mxb = -INFINITY;
+                        for (int c = 0; c < 64; ++c)
+                            if (c > tl) sreg[c] = 0xff800000u;   // -inf
+                    }
+                    if (i == 0 || pass == 1) {
+                        float mxa = -INFINITY, mxb = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 64; c += 4) {
-                    mxa = fmax3(mxa, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
-                    mxb = fmax3(mxb, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
-                }
-                const float mx = fmaxf(mxa, mxb);
-                if (i == 0) {
-                    m_used = mx;
-                } else {
-                    // The warp enters the branch together (the tensor-memory accesses in it are
-                    // warp-wide), but whether a row moves its reference maximum is that row's own
-                    // decision: a row that does not need it multiplies by exactly 1, so its
-                    // arithmetic never depends on the other rows of the warp (later tokens).
-                    const bool need = (mx - m_used) * c2 > kRescaleThreshold;
-                    if (__any_sync(0xffffffffu, need)) {
-                        const float alpha = need ? ex2_approx((m_used - mx) * c2) : 1.0f;
-                        l_run *= alpha;
-                        m_used = need ? mx : m_used;
-                        // O holds the sum up to tile i-1 once PV(g-1) has completed
-                        mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
-                        tc_fence_after();
+                        for (int c = 0; c < 64; c += 4) {
+                            mxa = fmax3(mxa, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+                            mxb = fmax3(mxb, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+                        }
+                        const float mx = fmaxf(mxa, mxb);
+                        if (i == 0) {
+                            m_used = mx;
+                        } else {
+                            const float alpha = tripped ? ex2_approx((m_used - mx) * c2) : 1.0f;
+                            l_run *= alpha;
+                            m_used = tripped ? mx : m_used;
+                            // O holds the sum up to tile i-1 once PV(g-1) has completed
+                            mbar_wait(bar_pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, args.status);
+                            tc_fence_after();
 #pragma unroll
-                        for (int c = 0; c < D / 16; ++c) {
-                            uint32_t oreg[16];
-                            tmem_ld16(t_lane + C::kColO + c * 16, oreg);
-                            tmem_wait_ld();
+                            for (int c = 0; c < D / 16; ++c) {
+                                uint32_t oreg[16];
+                                tmem_ld16(t_lane + C::kColO + c * 16, oreg);
+                                tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
-                            tmem_st16(t_lane + C::kColO + c * 16, oreg);
+                                for (int e = 0; e < 16; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
+                                tmem_st16(t_lane + C::kColO + c * 16, oreg);
+                            }
                         }
                     }
-                }
-                const float msc = m_used * c2;
-                const uint64_t c2p = pack2(c2, c2), mscp = pack2(-msc, -msc);
-                uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-                uint32_t preg[32];
+                    const float msc = m_used * c2;
+                    const uint64_t c2p = pack2(c2, c2), mscp = pack2(-msc, -msc);
+                    uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const uint64_t x = fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2p, mscp);
-                    float x0, x1;
-                    unpack2(x, x0, x1);
-                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                    if (c & 1) sum_b = add2(sum_b, pack2(p0, p1)); else sum_a = add2(sum_a, pack2(p0, p1));
-                    preg[c] = pack_bf16x2(p0, p1);
+                    for (int c = 0; c < 32; ++c) {
+                        const uint64_t x = fma2(pack2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])), c2p, mscp);
+                        float x0, x1;
+                        unpack2(x, x0, x1);
+                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                        if (c & 1) sum_b = add2(sum_b, pack2(p0, p1)); else sum_a = add2(sum_a, pack2(p0, p1));
+                        preg[c] = pack_bf16x2(p0, p1);
+                    }
+                    float r0, r1;
+                    unpack2(add2(sum_a, sum_b), r0, r1);
+                    tile_sum = r0 + r1;
+                    if (i == 0 || pass == 1) break;
+                    tripped = !(tile_sum < kSumGuard);
+                    if (!__any_sync(0xffffffffu, tripped)) break;
                 }
-                float r0, r1;
-                unpack2(add2(sum_a, sum_b), r0, r1);
-                l_run += r0 + r1;
+                l_run += tile_sum;
                 tmem_st32(t_s, preg);   // P overwrites the first 32 columns of this S buffer
                 tmem_wait_st();
                 tc_fence_before();

@@ -95,11 +95,12 @@ def test_future_token_isolation_is_bitwise():
 @pytest.mark.parametrize("dense", [False, True], ids=["bf1", "dense"])
 @pytest.mark.parametrize("hq,hkv", [(4, 2), (8, 2)], ids=["G2", "G4"])
 def test_future_token_isolation_is_bitwise_when_later_rows_rescale(dense, hq, hkv):
-    """The same gate on the path where it could fail: the kernel rescales a row's accumulator only
-    when that row's maximum jumps by more than 2^8 between tiles, and the rows of one warp are
-    consecutive tokens.  The mutated tokens get Q and K rows 36x larger, so that they jump in nearly
-    every tile while the untouched rows never do; t sits in the middle of a 32-row group, so untouched
-    and mutated rows share a warp.  Rows up to t must not change in a single bit."""
+    """The same gate on the path where it could fail: the kernel moves a row's reference maximum (and
+    rescales its accumulator) only when that row's exponentials outgrow the guard, the whole warp then
+    goes through the second pass together, and the rows of one warp are consecutive tokens.  The
+    mutated tokens get Q and K rows 36x larger, so that they overflow in nearly every tile while the
+    untouched rows never do; t sits in the middle of a 32-row group, so untouched and mutated rows
+    share a warp.  Rows up to t must not change in a single bit."""
     n = 600
     w = I.custom([n], hq=hq, hkv=hkv, d=128, seed=650 + hq)
     q, k, v = I.draw_qkv(w)
