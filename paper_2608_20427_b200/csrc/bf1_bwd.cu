@@ -69,6 +69,7 @@ struct BwdArgs {
     const int32_t* num_qblocks;
     const int32_t* order;      // may be null
     int32_t max_degree, capacity, total_tokens, hq, hkv, group;
+    int32_t interleave;    // 1: units of all KV heads interleaved (longest first over all heads); 0: KV head by KV head
     int32_t* status;
     float scale, scale_log2;
     const __nv_bfloat16* o;
@@ -231,10 +232,19 @@ __device__ __forceinline__ DqUnit dq_unit(const BwdArgs& a, int n, int nqb, int 
     u.cnt = 1;
     u.rows_valid = 0;
     if (u.ok) {
-        u.kvh = i / per_head;
-        const int rem = i - u.kvh * per_head;
-        const int rank = rem / pairs;
-        u.pair = rem - rank * pairs;
+        int rank;
+        if (a.interleave) {          // rank-major: the longest lists of all heads first
+            const int per_rank = pairs * a.hkv;
+            rank = i / per_rank;
+            const int rem = i - rank * per_rank;
+            u.kvh = rem / pairs;
+            u.pair = rem - u.kvh * pairs;
+        } else {                     // head-major: a head's K and V stay hot in L2
+            u.kvh = i / per_head;
+            const int rem = i - u.kvh * per_head;
+            rank = rem / pairs;
+            u.pair = rem - rank * pairs;
+        }
         int slot = a.order ? a.order[rank] : rank;
         slot = min(max(slot, 0), nqb - 1);
         u.slot = slot;
@@ -795,8 +805,15 @@ __device__ __forceinline__ DkvUnit dkv_unit(const BwdArgs& a, int n, int n_units
     u.steps = 0;
     u.part = -1;
     if (u.ok) {
-        u.kvh = i / n_units;
-        const int unit = a.inv.unit_order[i - u.kvh * n_units];
+        int ui;
+        if (a.interleave) {
+            ui = i / a.hkv;
+            u.kvh = i - ui * a.hkv;
+        } else {
+            u.kvh = i / n_units;
+            ui = i - u.kvh * n_units;
+        }
+        const int unit = a.inv.unit_order[ui];
         u.gp = a.inv.unit_slot[unit];
         u.r_begin = a.inv.unit_begin[unit];
         u.steps = (a.inv.unit_end[unit] - u.r_begin) * pairs;
@@ -1199,6 +1216,9 @@ extern "C" int bf1_attn_bwd(const void* q, const void* k, const void* v, const v
     a.status = route->status;
     a.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)d);
     a.scale_log2 = a.scale * 1.4426950408889634f;
+    // The same rule as the forward's hand-out order: while K and V of all heads fit L2 together there is nothing
+    // to gain from working head by head, and the longest units of all heads first balance the CTAs better.
+    a.interleave = (total_tokens * (int64_t)hkv * d * 4 <= (48LL << 20)) ? 1 : 0;
     a.o = (const __nv_bfloat16*)o;
     a.d_o = (const __nv_bfloat16*)d_o;
     a.lse = lse;
