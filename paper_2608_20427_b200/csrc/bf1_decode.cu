@@ -93,11 +93,15 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
     __shared__ float sW[2][64];                         // combine: weight of every partial
     __shared__ float sRed[2][2];
     __shared__ int sLast;
+    __shared__ int sPages[64];                          // the sequence's page list (max_degree <= 64)
 
     const int kvp = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
     const int kvh = kvp / a.pairs, hbase = kvh * a.group + (kvp % a.pairs) * 2;   // first query head of this CTA's pair
     const int nheads = min(2, a.group - (kvp % a.pairs) * 2);                      // 1 when G = 1
     const int warp = tid >> 5, lane = tid & 31, gid = lane >> 2, tig = lane & 3;
+    // The page list is fetched together with the plan's count and the length (independent loads in flight at
+    // once), not after them: at small batch the kernel is one chain of dependent memory round trips.
+    if (tid < a.max_degree) sPages[tid] = a.page[(size_t)s * a.max_degree + tid];
     const int cnt = a.count[s];
     const int n = a.seqlens[s];
     if (cnt <= 0) return;
@@ -107,7 +111,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_fused_kernel(const DecodeA
         return;
     }
     const int tail = n - j * kPage;   // valid tokens of the self page (the last list entry)
-    const int32_t* pages = a.page + (size_t)s * a.max_degree;
+    __syncthreads();                  // sPages is complete (every exit above is taken by the whole CTA)
+    const int* pages = sPages;
     // the part of the list this CTA walks: all of it, or the z-th run of `per` entries
     const int per = kSplit ? (cnt + a.nsplit - 1) / a.nsplit : cnt;
     const int e_lo = kSplit ? (int)blockIdx.z * per : 0, e_hi = min(cnt, e_lo + per);
