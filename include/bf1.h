@@ -127,9 +127,10 @@ int bf1_plan_route(const int32_t *cu_seqlens_dev, int32_t batch, int64_t total_t
  * the KV blocks its list names, causal triangle on the self block.
  *   q, k, v   device bf16, [T, hq, d], [T, hkv, d], [T, hkv, d]
  *   softmax_scale  scores are scale * <q, k>; <= 0 selects 1 / sqrt(d)
- *   route     a route planned for the same cu_seqlens (any ascending lists whose last
- *             entry is the query block itself are accepted, so other block-sparse causal
- *             routes can be run through the same kernel)
+ *   route     a route planned for the same cu_seqlens (any lists of distinct earlier blocks
+ *             whose last entry is the query block itself are accepted, so other block-sparse
+ *             causal routes can be run through the same kernel; the planners write the
+ *             earlier blocks in ascending order, the kernel does not depend on it)
  *   o         device bf16 [T, hq, d], written for every token row
  *   lse       device fp32 [hq, T]: natural log of the sum of exp(scaled scores) over the
  *             selected keys
@@ -274,6 +275,24 @@ int bf1_plan_route_shard(int64_t n_tokens, int32_t lo_block, int32_t hi_block,
                          const bf1_route_cfg *cfg /* host */, const int32_t *needed_blocks_dev,
                          int32_t num_needed, const bf1_route *out /* host struct, device arrays */,
                          int32_t *cu_seqlens_out_dev /* [2] */, void *stream);
+
+/* The same two plans for a shard that owns every `stride`-th block: first_block, first_block + stride, ...,
+ * num_blocks of them (rank r of R ranks: first_block = r, stride = R).  The route is block aligned and data
+ * independent (Section 3.1) and its long edges are powers of two (Eq. 1), so with a power-of-two stride the dyadic
+ * predecessors j - 2^k with 2^k >= stride of an owned block are owned as well: a rank is sent little more than the
+ * window in front of each of its blocks and block 0 (about two blocks per own block, whatever its rank), and all
+ * ranks hold lists of the same lengths -- where contiguous shards leave the first rank with the short lists and
+ * send the last one most of the sequence.  The local key/value tensor is laid out as before, [the needed blocks in
+ * ascending global order | the own blocks in ascending order]; a list is re-indexed entry by entry, so its local
+ * indices end in the query block itself but need not ascend (the attention kernel does not require it). */
+int bf1_shard_needed_blocks_strided(int64_t n_tokens, const bf1_route_cfg *cfg /* host */, int32_t first_block,
+                                    int32_t stride, int32_t num_blocks, int32_t *blocks_out /* host */,
+                                    int32_t capacity, int32_t *count_out /* host */);
+int bf1_plan_route_shard_strided(int64_t n_tokens, int32_t first_block, int32_t stride, int32_t num_blocks,
+                                 const bf1_route_cfg *cfg /* host */, const int32_t *needed_blocks_dev,
+                                 int32_t num_needed, const bf1_route *out /* host struct, device arrays */,
+                                 int32_t *cu_seqlens_out_dev, void *stream);
+
 
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char *bf1_last_error(void);

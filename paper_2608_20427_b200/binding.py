@@ -21,6 +21,7 @@ DEV_BAD_SEQLENS, DEV_CAPACITY, DEV_WAIT_TIMEOUT, DEV_BAD_ROUTE = 1, 2, 4, 8
 EXPORTS = ("bf1_route_capacity", "bf1_plan_route", "bf1_attn_fwd", "bf1_dense_causal_fwd",
            "bf1_attn_fwd_noalloc", "bf1_plan_decode", "bf1_decode_workspace_bytes", "bf1_decode_fwd",
            "bf1_attn_bwd", "bf1_attn_bwd_workspace_bytes", "bf1_shard_needed_blocks", "bf1_plan_route_shard",
+           "bf1_shard_needed_blocks_strided", "bf1_plan_route_shard_strided",
            "bf1_last_error", "bf1_version")
 
 
@@ -93,6 +94,12 @@ def load():
     L.bf1_shard_needed_blocks.argtypes = [i64, ctypes.POINTER(RouteCfg), i32, i32, ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
     L.bf1_plan_route_shard.restype = ctypes.c_int
     L.bf1_plan_route_shard.argtypes = [i64, i32, i32, ctypes.POINTER(RouteCfg), vp, i32, ctypes.POINTER(_RouteC), vp, vp]
+    L.bf1_shard_needed_blocks_strided.restype = ctypes.c_int
+    L.bf1_shard_needed_blocks_strided.argtypes = [i64, ctypes.POINTER(RouteCfg), i32, i32, i32, ctypes.POINTER(i32), i32,
+                                                  ctypes.POINTER(i32)]
+    L.bf1_plan_route_shard_strided.restype = ctypes.c_int
+    L.bf1_plan_route_shard_strided.argtypes = [i64, i32, i32, i32, ctypes.POINTER(RouteCfg), vp, i32, ctypes.POINTER(_RouteC),
+                                               vp, vp]
     L.bf1_last_error.restype = ctypes.c_char_p
     L.bf1_last_error.argtypes = []
     L.bf1_version.restype = ctypes.c_int
@@ -353,6 +360,40 @@ def plan_route_shard(n_tokens: int, lo_block: int, hi_block: int, needed_blocks:
                                        needed_blocks.data_ptr() if needed_blocks.numel() else None, needed_blocks.numel(),
                                        ctypes.byref(route.c), cu.data_ptr(), _stream_ptr(stream)))
     own_tokens = min(n_tokens, hi_block * 64) - lo_block * 64
+    cu._bf1_total = needed_blocks.numel() * 64 + own_tokens
+    route.cfg = cfg
+    return route, cu
+
+
+def shard_needed_blocks_strided(n_tokens: int, first_block: int, stride: int, num_blocks: int,
+                                cfg: Optional[RouteCfg] = None):
+    """bf1_shard_needed_blocks_strided: ascending global KV blocks read but not owned by the shard
+    first_block, first_block + stride, ... (num_blocks of them); host only."""
+    cfg = cfg or RouteCfg()
+    cap = max(first_block + (num_blocks - 1) * stride, 1)
+    buf = (ctypes.c_int32 * cap)()
+    count = ctypes.c_int32(0)
+    _check(load().bf1_shard_needed_blocks_strided(n_tokens, ctypes.byref(cfg), first_block, stride, num_blocks, buf, cap,
+                                                  ctypes.byref(count)))
+    return list(buf[:count.value])
+
+
+def plan_route_shard_strided(n_tokens: int, first_block: int, stride: int, num_blocks: int, needed_blocks: torch.Tensor,
+                             cfg: Optional[RouteCfg] = None, route: Optional[Route] = None, stream=None):
+    """bf1_plan_route_shard_strided: the strided shard's route over its local [needed | own] key/value tensor.
+    Returns (route, cu_seqlens [2] int32 device tensor of the shard's virtual sequence)."""
+    cfg = cfg or RouteCfg()
+    assert needed_blocks.dtype == torch.int32 and needed_blocks.is_cuda
+    if route is None:
+        _, deg = route_capacity(1, n_tokens, n_tokens, cfg)
+        route = Route.empty(num_blocks, deg, needed_blocks.device, cfg)
+    cu = torch.zeros(2, dtype=torch.int32, device=needed_blocks.device)
+    _check(load().bf1_plan_route_shard_strided(n_tokens, first_block, stride, num_blocks, ctypes.byref(cfg),
+                                               needed_blocks.data_ptr() if needed_blocks.numel() else None,
+                                               needed_blocks.numel(), ctypes.byref(route.c), cu.data_ptr(),
+                                               _stream_ptr(stream)))
+    last = first_block + (num_blocks - 1) * stride
+    own_tokens = (num_blocks - 1) * 64 + min(64, n_tokens - last * 64)
     cu._bf1_total = needed_blocks.numel() * 64 + own_tokens
     route.cfg = cfg
     return route, cu

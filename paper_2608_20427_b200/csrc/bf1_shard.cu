@@ -8,6 +8,9 @@
 //
 //   bf1_shard_needed_blocks   host: which blocks the shard reads but does not own
 //   bf1_plan_route_shard      device: the shard's route over its local [needed | own] key/value tensor
+// A shard may also own every `stride`-th block (the *_strided entry points): with a power-of-two stride the dyadic
+// predecessors j - 2^k, 2^k >= stride, of an owned block are owned too, so that every rank is sent about two
+// blocks per block of its own (the window in front of each) and all ranks carry the same work.
 #include "bf1_common.cuh"
 
 namespace bf1 {
@@ -44,12 +47,23 @@ __host__ __device__ inline int for_each_selected(const bf1_route_cfg& c, int j, 
     return deg;
 }
 
-// Host side: marks the selected blocks in front of `limit` in a bitmap.
-struct MarkInFront {
+// The blocks a shard owns: first, first + stride, ..., `count` of them (stride 1: a contiguous range).
+struct Owned {
+    int first, stride, count;
+    __host__ __device__ bool has(int p) const {
+        const int off = p - first;
+        return off >= 0 && off % stride == 0 && off / stride < count;
+    }
+    __host__ __device__ int index(int p) const { return (p - first) / stride; }   // only for owned blocks
+    __host__ __device__ int block(int g) const { return first + g * stride; }
+};
+
+// Host side: marks the selected blocks that the shard does not own in a bitmap.
+struct MarkNotOwned {
     uint64_t* seen;
-    int limit;
+    Owned own;
     __host__ __device__ void operator()(int p, int) {
-        if (p < limit) seen[p >> 6] |= 1ull << (p & 63);
+        if (!own.has(p)) seen[p >> 6] |= 1ull << (p & 63);
     }
 };
 
@@ -57,12 +71,14 @@ struct MarkInFront {
 struct WriteLocalEntry {
     int32_t* list;
     const int32_t* needed;
-    int num_needed, lo_block, max_degree;
+    int num_needed;
+    Owned own;
+    int max_degree;
     int bad;
     __device__ void operator()(int p, int pos) {
         int idx;
-        if (p >= lo_block) {
-            idx = num_needed + (p - lo_block);             // an own block: behind the landing area
+        if (own.has(p)) {
+            idx = num_needed + own.index(p);               // an own block: behind the landing area
         } else {
             int lo = 0, hi = num_needed;                    // a received block: its place in the ascending list
             while (lo < hi) {
@@ -81,7 +97,8 @@ struct WriteLocalEntry {
 
 struct ShardArgs {
     int64_t n_tokens;
-    int32_t lo, hi, num_needed;
+    Owned own;
+    int32_t num_needed;
     const int32_t* needed;
     bf1_route_cfg cfg;
     bf1_route route;
@@ -97,7 +114,7 @@ __global__ void __launch_bounds__(kShardThreads, 1) plan_shard_kernel(const Shar
     const int tid = threadIdx.x;
     const bf1_route& r = a.route;
     const int b = a.cfg.block;
-    const int nloc = a.hi - a.lo;
+    const int nloc = a.own.count;
     if (tid == 0) {
         s_bad = 0;
         s_total = 0ull;
@@ -120,11 +137,11 @@ __global__ void __launch_bounds__(kShardThreads, 1) plan_shard_kernel(const Shar
     }
     unsigned long long my_pairs = 0ull;
     for (int g = tid; g < nloc; g += kShardThreads) {
-        const int j = a.lo + g;
+        const int j = a.own.block(g);
         const long long left = a.n_tokens - (long long)j * b;
         const int rows = left < b ? (int)left : b;
         int32_t* list = r.kv_idx + (size_t)g * r.max_degree;
-        WriteLocalEntry w{list, a.needed, a.num_needed, a.lo, r.max_degree, 0};
+        WriteLocalEntry w{list, a.needed, a.num_needed, a.own, r.max_degree, 0};
         const int deg = for_each_selected(a.cfg, j, w);
         if (w.bad) atomicOr(&s_bad, w.bad);
         const int kept = deg < r.max_degree ? deg : r.max_degree;
@@ -156,7 +173,9 @@ __global__ void __launch_bounds__(kShardThreads, 1) plan_shard_kernel(const Shar
         r.order[pos] = g;
     }
     if (tid == 0) {
-        const long long own_tokens = (a.n_tokens < (long long)a.hi * b ? a.n_tokens : (long long)a.hi * b) - (long long)a.lo * b;
+        // every owned block but the last is full (it precedes another block of the sequence)
+        const long long last_left = a.n_tokens - (long long)a.own.block(nloc - 1) * b;
+        const long long own_tokens = (long long)(nloc - 1) * b + (last_left < b ? last_left : b);
         *r.status = s_bad;
         *r.num_qblocks = s_bad ? 0 : nloc;
         *r.total_pairs = (int64_t)s_total;
@@ -167,33 +186,30 @@ __global__ void __launch_bounds__(kShardThreads, 1) plan_shard_kernel(const Shar
     }
 }
 
-static int check_shard(int64_t n_tokens, const bf1_route_cfg* cfg, int32_t lo_block, int32_t hi_block) {
+// A shard is `count` blocks first, first + stride, ... of a sequence of n_tokens tokens.
+static int check_shard(int64_t n_tokens, const bf1_route_cfg* cfg, int32_t first, int32_t stride, int32_t count) {
     if (int rc = check_cfg(cfg)) return rc;
     if (cfg->block != 64) return fail(BF1_ERR_UNSUPPORTED, "sequence sharding is built for b = 64 only (block width %d)", cfg->block);
     if (n_tokens < 1 || n_tokens > 0x7fffffffLL - 64) return fail(BF1_ERR_INVALID_ARG, "n_tokens %lld out of range", (long long)n_tokens);
     const int64_t nb = (n_tokens + cfg->block - 1) / cfg->block;
-    if (lo_block < 0 || hi_block <= lo_block || hi_block > nb)
-        return fail(BF1_ERR_INVALID_ARG, "shard blocks [%d, %d) are not inside the sequence's %lld blocks", lo_block, hi_block,
-                    (long long)nb);
+    if (first < 0 || stride < 1 || count < 1 || (int64_t)first + (int64_t)(count - 1) * stride >= nb)
+        return fail(BF1_ERR_INVALID_ARG, "shard blocks %d + k * %d, k < %d, are not inside the sequence's %lld blocks", first,
+                    stride, count, (long long)nb);
     return BF1_OK;
 }
 
-}  // namespace bf1
-
-using namespace bf1;
-
-extern "C" int bf1_shard_needed_blocks(int64_t n_tokens, const bf1_route_cfg* cfg, int32_t lo_block, int32_t hi_block,
-                                       int32_t* blocks_out, int32_t capacity, int32_t* count_out) {
-    if (int rc = check_shard(n_tokens, cfg, lo_block, hi_block)) return rc;
+static int needed_blocks(int64_t n_tokens, const bf1_route_cfg* cfg, const Owned& own, int32_t* blocks_out,
+                         int32_t capacity, int32_t* count_out) {
     if (!count_out || capacity < 0 || (capacity > 0 && !blocks_out)) return fail(BF1_ERR_INVALID_ARG, "output pointer is null");
-    // every needed block is < lo_block: mark them in a bitmap over [0, lo_block), then read it out in order
-    const size_t words = ((size_t)lo_block + 63) / 64;
+    // every needed block lies in front of the shard's last block: mark them in a bitmap, then read it out in order
+    const int last = own.block(own.count - 1);
+    const size_t words = ((size_t)last + 63) / 64;
     uint64_t* seen = words ? (uint64_t*)calloc(words, sizeof(uint64_t)) : nullptr;
     if (words && !seen) return fail(BF1_ERR_INVALID_ARG, "out of host memory");
-    MarkInFront mark{seen, lo_block};
-    for (int j = lo_block; j < hi_block; ++j) for_each_selected(*cfg, j, mark);
+    MarkNotOwned mark{seen, own};
+    for (int g = 0; g < own.count; ++g) for_each_selected(*cfg, own.block(g), mark);
     int32_t count = 0;
-    for (int p = 0; p < lo_block; ++p)
+    for (int p = 0; p < last; ++p)
         if (seen[p >> 6] >> (p & 63) & 1) {
             if (count < capacity) blocks_out[count] = p;
             ++count;
@@ -204,26 +220,23 @@ extern "C" int bf1_shard_needed_blocks(int64_t n_tokens, const bf1_route_cfg* cf
     return BF1_OK;
 }
 
-extern "C" int bf1_plan_route_shard(int64_t n_tokens, int32_t lo_block, int32_t hi_block, const bf1_route_cfg* cfg,
-                                    const int32_t* needed_blocks_dev, int32_t num_needed, const bf1_route* out,
-                                    int32_t* cu_seqlens_out_dev, void* stream) {
-    if (int rc = check_shard(n_tokens, cfg, lo_block, hi_block)) return rc;
+static int plan_shard(int64_t n_tokens, const Owned& own, const bf1_route_cfg* cfg, const int32_t* needed_blocks_dev,
+                      int32_t num_needed, const bf1_route* out, int32_t* cu_seqlens_out_dev, void* stream) {
     if (!out || !cu_seqlens_out_dev || num_needed < 0 || (num_needed > 0 && !needed_blocks_dev))
         return fail(BF1_ERR_INVALID_ARG, "route, cu_seqlens_out or needed_blocks is null");
     if (!out->qb_seq || !out->qb_block || !out->kv_count || !out->kv_idx || !out->pair_count || !out->order ||
         !out->total_pairs || !out->num_qblocks || !out->status || !out->sched)
         return fail(BF1_ERR_INVALID_ARG, "a route array pointer is null");
-    if (out->capacity_qblocks < hi_block - lo_block)
+    if (out->capacity_qblocks < own.count)
         return fail(BF1_ERR_CAPACITY, "route capacity_qblocks %d < %d query blocks of the shard", out->capacity_qblocks,
-                    hi_block - lo_block);
+                    own.count);
     int32_t cap = 0, need_deg = 0;
     if (int rc = bf1_route_capacity(1, n_tokens, (int32_t)n_tokens, cfg, &cap, &need_deg)) return rc;
     if (out->max_degree < need_deg || out->max_degree > 64)
         return fail(BF1_ERR_CAPACITY, "route max_degree %d: need %d .. 64", out->max_degree, need_deg);
     ShardArgs a;
     a.n_tokens = n_tokens;
-    a.lo = lo_block;
-    a.hi = hi_block;
+    a.own = own;
     a.num_needed = num_needed;
     a.needed = needed_blocks_dev;
     a.cfg = *cfg;
@@ -232,4 +245,40 @@ extern "C" int bf1_plan_route_shard(int64_t n_tokens, int32_t lo_block, int32_t 
     plan_shard_kernel<<<1, kShardThreads, 0, (cudaStream_t)stream>>>(a);
     BF1_CUDA_CHECK(cudaGetLastError());
     return BF1_OK;
+}
+
+}  // namespace bf1
+
+using namespace bf1;
+
+extern "C" int bf1_shard_needed_blocks(int64_t n_tokens, const bf1_route_cfg* cfg, int32_t lo_block, int32_t hi_block,
+                                       int32_t* blocks_out, int32_t capacity, int32_t* count_out) {
+    if (hi_block <= lo_block) return fail(BF1_ERR_INVALID_ARG, "shard blocks [%d, %d) are empty", lo_block, hi_block);
+    if (int rc = check_shard(n_tokens, cfg, lo_block, 1, hi_block - lo_block)) return rc;
+    return needed_blocks(n_tokens, cfg, Owned{lo_block, 1, hi_block - lo_block}, blocks_out, capacity, count_out);
+}
+
+extern "C" int bf1_plan_route_shard(int64_t n_tokens, int32_t lo_block, int32_t hi_block, const bf1_route_cfg* cfg,
+                                    const int32_t* needed_blocks_dev, int32_t num_needed, const bf1_route* out,
+                                    int32_t* cu_seqlens_out_dev, void* stream) {
+    if (hi_block <= lo_block) return fail(BF1_ERR_INVALID_ARG, "shard blocks [%d, %d) are empty", lo_block, hi_block);
+    if (int rc = check_shard(n_tokens, cfg, lo_block, 1, hi_block - lo_block)) return rc;
+    return plan_shard(n_tokens, Owned{lo_block, 1, hi_block - lo_block}, cfg, needed_blocks_dev, num_needed, out,
+                      cu_seqlens_out_dev, stream);
+}
+
+extern "C" int bf1_shard_needed_blocks_strided(int64_t n_tokens, const bf1_route_cfg* cfg, int32_t first_block,
+                                               int32_t stride, int32_t num_blocks, int32_t* blocks_out,
+                                               int32_t capacity, int32_t* count_out) {
+    if (int rc = check_shard(n_tokens, cfg, first_block, stride, num_blocks)) return rc;
+    return needed_blocks(n_tokens, cfg, Owned{first_block, stride, num_blocks}, blocks_out, capacity, count_out);
+}
+
+extern "C" int bf1_plan_route_shard_strided(int64_t n_tokens, int32_t first_block, int32_t stride, int32_t num_blocks,
+                                            const bf1_route_cfg* cfg, const int32_t* needed_blocks_dev,
+                                            int32_t num_needed, const bf1_route* out, int32_t* cu_seqlens_out_dev,
+                                            void* stream) {
+    if (int rc = check_shard(n_tokens, cfg, first_block, stride, num_blocks)) return rc;
+    return plan_shard(n_tokens, Owned{first_block, stride, num_blocks}, cfg, needed_blocks_dev, num_needed, out,
+                      cu_seqlens_out_dev, stream);
 }
